@@ -1,0 +1,409 @@
+/*
+ * CPU oracle for the multi-coil SENSE data-consistency step  (TEST INFRASTRUCTURE).
+ *
+ * This file is test infrastructure only.  It is a slow, double-precision, obviously-correct
+ * evaluation of the definitions in the GLEAM paper (arXiv 2207.08393).  It shares no code,
+ * header, table or constant generator with the CUDA library, and the CUDA library never calls it.
+ *
+ *   Sensing model (Eq. 1):          y = Omega F S x + eps
+ *   Forward operator (after Eq. 2): A = Omega F S ,  A^H its Hermitian transpose
+ *   Data-consistency step (Eq. 3):  DC(x) = x - 2t A^H (A x - y)         (eta := 2t)
+ *   Its vector-Jacobian product:    J^H g = g - eta A^H A g              (J = I - eta A^H A)
+ *
+ * Conventions the paper leaves open ("F is the Fourier transform matrix") and that are fixed
+ * here:  F is the centred, orthonormal DFT over the trailing fft_rank spatial axes,
+ *
+ *      X[k] = N^(-1/2) * sum_n x[n] * exp(-2 pi i (k - o)(n - o) / N),    o = floor(N / 2),
+ *
+ * applied separably along every transformed axis; F^H uses +2 pi i.  Omega is a real diagonal
+ * weight (normally 0/1) and is applied literally once in A and once in A^H:
+ *      r_c = M .* (M .* F(S_c .* x) - y_c).
+ *
+ * Layout (row-major, last index fastest):
+ *      x, out : (B, T, n0, n1, n2)           complex
+ *      y      : (B, C, T, n0, n1, n2)        complex
+ *      sens   : (B, C, n0, n1, n2)  or  (B, C, T, n0, n1, n2)   (sens_has_frames)
+ *      mask   : mask_kind 0: (B, T, n0, n1, n2) real
+ *               mask_kind 1: readout-invariant; fft_rank 2 -> (B, T, n2),  fft_rank 3 -> (B, T, n1, n2)
+ * n0 = 1 when fft_rank == 2.  The frame axis T is never transformed.
+ *
+ * Inputs are single precision (the arrays the GPU sees), promoted to double; outputs are double.
+ *
+ * Pins (tests/test_oracle_pins.py): brute-force DFT, closed-form spectra of deltas and
+ * constants, Parseval, adjoint identity, Hermitian/PSD normal operator, A^H A = I for a full mask
+ * and unit-norm sensitivities, affine structure, an independent library FFT.
+ */
+#include <complex.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef double complex zc;
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG (-1)
+#define ORACLE_ERR_MEM (-2)
+
+static const double TWO_PI = 6.283185307179586476925286766559;
+
+/* ------------------------------------------------------------------------------------------
+ * 1-D transforms
+ * ---------------------------------------------------------------------------------------- */
+
+/* The definition itself, by direct summation.  sign = -1: F (image -> k-space); +1: F^H.
+ * The phase index (k-o)(n-o) is reduced modulo N in integers so that the argument of exp stays
+ * in [0, 2 pi). */
+void oracle_dft_naive_1d(const zc* in, zc* out, int64_t N, int sign)
+{
+    const int64_t o = N / 2;
+    const double scale = 1.0 / sqrt((double)N);
+    for (int64_t k = 0; k < N; ++k) {
+        zc acc = 0.0;
+        for (int64_t n = 0; n < N; ++n) {
+            int64_t p = ((k - o) * (n - o)) % N;
+            if (p < 0) p += N;
+            const double ang = sign * TWO_PI * (double)p / (double)N;
+            acc += in[n] * (cos(ang) + I * sin(ang));
+        }
+        out[k] = acc * scale;
+    }
+}
+
+/* Raw (uncentred, unscaled) DFT of a strided sequence: halve while the length is even
+ * (decimation in time), evaluate the odd remainder by direct summation.
+ * tw[j] = exp(sign 2 pi i j / N_top); at this level the root of unity is tw[tws]. */
+static void fft_rec(const zc* in, int64_t stride, zc* out, int64_t n, const zc* tw, int64_t tws)
+{
+    if (n == 1) { out[0] = in[0]; return; }
+    if (n % 2 != 0) {
+        for (int64_t k = 0; k < n; ++k) {
+            zc acc = 0.0;
+            for (int64_t j = 0; j < n; ++j) acc += in[j * stride] * tw[((j * k) % n) * tws];
+            out[k] = acc;
+        }
+        return;
+    }
+    const int64_t h = n / 2;
+    fft_rec(in, 2 * stride, out, h, tw, 2 * tws);
+    fft_rec(in + stride, 2 * stride, out + h, h, tw, 2 * tws);
+    for (int64_t k = 0; k < h; ++k) {
+        const zc e = out[k];
+        const zc t = tw[k * tws] * out[k + h];
+        out[k] = e + t;
+        out[k + h] = e - t;
+    }
+}
+
+/* Centred orthonormal transform: ifftshift -> raw FFT -> fftshift -> 1/sqrt(N).
+ * Lengths up to 32 go through the direct sum.  work must hold 2 N entries, tw N entries
+ * (tw[j] = exp(sign 2 pi i j / N)). */
+static void fft_centered_line(const zc* in, zc* out, int64_t N, int sign, zc* work, const zc* tw)
+{
+    if (N <= 32) { oracle_dft_naive_1d(in, out, N, sign); return; }
+    const int64_t o = N / 2;
+    zc* a = work;
+    zc* b = work + N;
+    for (int64_t j = 0; j < N; ++j) a[j] = in[(j + o) % N];
+    fft_rec(a, 1, b, N, tw, 1);
+    const double scale = 1.0 / sqrt((double)N);
+    for (int64_t j = 0; j < N; ++j) out[(j + o) % N] = b[j] * scale;
+}
+
+static zc* make_twiddles(int64_t N, int sign)
+{
+    zc* tw = (zc*)malloc(sizeof(zc) * (size_t)N);
+    if (!tw) return NULL;
+    for (int64_t j = 0; j < N; ++j) {
+        const double ang = sign * TWO_PI * (double)j / (double)N;
+        tw[j] = cos(ang) + I * sin(ang);
+    }
+    return tw;
+}
+
+int oracle_fft_centered_1d(const zc* in, zc* out, int64_t N, int sign)
+{
+    if (N < 1 || (sign != 1 && sign != -1)) return ORACLE_ERR_ARG;
+    zc* work = (zc*)malloc(sizeof(zc) * (size_t)(2 * N));
+    zc* tw = make_twiddles(N, sign);
+    if (!work || !tw) { free(work); free(tw); return ORACLE_ERR_MEM; }
+    fft_centered_line(in, out, N, sign, work, tw);
+    free(work); free(tw);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * N-D transform over the trailing `rank` axes of `outer` volumes of shape n[0..2], in place.
+ * ---------------------------------------------------------------------------------------- */
+static int fft_centered_volume(zc* data, const int64_t n[3], int rank, int sign)
+{
+    const int64_t V = n[0] * n[1] * n[2];
+    for (int ax = 3 - rank; ax < 3; ++ax) {
+        const int64_t N = n[ax];
+        if (N == 1) continue;
+        int64_t stride = 1;
+        for (int a = ax + 1; a < 3; ++a) stride *= n[a];
+        const int64_t nlines = V / N;
+        zc* tw = make_twiddles(N, sign);
+        zc* buf = (zc*)malloc(sizeof(zc) * (size_t)(4 * N));
+        if (!tw || !buf) { free(tw); free(buf); return ORACLE_ERR_MEM; }
+        for (int64_t l = 0; l < nlines; ++l) {
+            /* line l: all indices except axis ax */
+            const int64_t inner = l % stride;
+            const int64_t outerl = l / stride;
+            zc* base = data + outerl * stride * N + inner;
+            zc* li = buf;
+            zc* lo = buf + N;
+            for (int64_t j = 0; j < N; ++j) li[j] = base[j * stride];
+            fft_centered_line(li, lo, N, sign, buf + 2 * N, tw);
+            for (int64_t j = 0; j < N; ++j) base[j * stride] = lo[j];
+        }
+        free(tw); free(buf);
+    }
+    return ORACLE_OK;
+}
+
+/* Public: centred orthonormal DFT over the trailing `rank` axes of `outer` stacked volumes. */
+int oracle_fftn_centered(zc* data, int64_t outer, const int64_t n[3], int rank, int sign, int nthreads)
+{
+    if (rank < 1 || rank > 3 || outer < 0) return ORACLE_ERR_ARG;
+    const int64_t V = n[0] * n[1] * n[2];
+    int rc = ORACLE_OK;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(dynamic, 1)
+#endif
+    for (int64_t u = 0; u < outer; ++u) {
+        const int r = fft_centered_volume(data + u * V, n, rank, sign);
+        if (r != ORACLE_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            rc = r;
+        }
+    }
+    return rc;
+}
+
+/* The definition in N-D by direct summation along each axis (tiny inputs only). */
+int oracle_dftn_naive(zc* data, int64_t outer, const int64_t n[3], int rank, int sign)
+{
+    if (rank < 1 || rank > 3) return ORACLE_ERR_ARG;
+    const int64_t V = n[0] * n[1] * n[2];
+    for (int64_t u = 0; u < outer; ++u) {
+        zc* vol = data + u * V;
+        for (int ax = 3 - rank; ax < 3; ++ax) {
+            const int64_t N = n[ax];
+            int64_t stride = 1;
+            for (int a = ax + 1; a < 3; ++a) stride *= n[a];
+            zc* li = (zc*)malloc(sizeof(zc) * (size_t)(2 * N));
+            if (!li) return ORACLE_ERR_MEM;
+            zc* lo = li + N;
+            for (int64_t l = 0; l < V / N; ++l) {
+                zc* base = vol + (l / stride) * stride * N + (l % stride);
+                for (int64_t j = 0; j < N; ++j) li[j] = base[j * stride];
+                oracle_dft_naive_1d(li, lo, N, sign);
+                for (int64_t j = 0; j < N; ++j) base[j * stride] = lo[j];
+            }
+            free(li);
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * The operators.  `dims` = {B, C, T, fft_rank, n0, n1, n2, sens_has_frames, mask_kind}.
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t B, C, T;
+    int rank;
+    int64_t n[3];
+    int sens_has_frames;
+    int mask_kind;
+    int64_t V;
+} odims;
+
+static int parse_dims(const int64_t* d, odims* o)
+{
+    o->B = d[0]; o->C = d[1]; o->T = d[2]; o->rank = (int)d[3];
+    o->n[0] = d[4]; o->n[1] = d[5]; o->n[2] = d[6];
+    o->sens_has_frames = (int)d[7]; o->mask_kind = (int)d[8];
+    if (o->B < 1 || o->C < 1 || o->T < 1) return ORACLE_ERR_ARG;
+    if (o->rank != 2 && o->rank != 3) return ORACLE_ERR_ARG;
+    if (o->n[0] < 1 || o->n[1] < 1 || o->n[2] < 1) return ORACLE_ERR_ARG;
+    if (o->rank == 2 && o->n[0] != 1) return ORACLE_ERR_ARG;
+    if (o->mask_kind != 0 && o->mask_kind != 1) return ORACLE_ERR_ARG;
+    o->V = o->n[0] * o->n[1] * o->n[2];
+    return ORACLE_OK;
+}
+
+/* Omega at voxel p of example b, frame t (p = flat index into (n0,n1,n2)). */
+static inline double mask_at(const float* mask, const odims* o, int64_t b, int64_t t, int64_t p)
+{
+    if (o->mask_kind == 0) return (double)mask[(b * o->T + t) * o->V + p];
+    /* readout-invariant: depends on the phase-encode indices only */
+    if (o->rank == 2) return (double)mask[(b * o->T + t) * o->n[2] + (p % o->n[2])];
+    const int64_t pe = o->n[1] * o->n[2];
+    return (double)mask[(b * o->T + t) * pe + (p % pe)];
+}
+
+static inline const float* sens_ptr(const float* sens, const odims* o, int64_t b, int64_t c, int64_t t)
+{
+    const int64_t idx = o->sens_has_frames ? ((b * o->C + c) * o->T + t) : (b * o->C + c);
+    return sens + 2 * idx * o->V;
+}
+
+/* k = A x  (Eq. 1 without noise):  k[b,c,t] = M .* F(S_c .* x).   k: (B,C,T,V) double complex. */
+int oracle_apply_A(const float* x, const float* sens, const float* mask, const int64_t* dims,
+                   zc* k, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK) return ORACLE_ERR_ARG;
+    int rc = ORACLE_OK;
+    const int64_t units = o.B * o.C * o.T;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(dynamic, 1)
+#endif
+    for (int64_t u = 0; u < units; ++u) {
+        const int64_t t = u % o.T, c = (u / o.T) % o.C, b = u / (o.T * o.C);
+        const float* xs = x + 2 * (b * o.T + t) * o.V;
+        const float* ss = sens_ptr(sens, &o, b, c, t);
+        zc* ku = k + u * o.V;
+        for (int64_t p = 0; p < o.V; ++p) {
+            const zc xv = (double)xs[2 * p] + I * (double)xs[2 * p + 1];
+            const zc sv = (double)ss[2 * p] + I * (double)ss[2 * p + 1];
+            ku[p] = sv * xv;
+        }
+        const int r = fft_centered_volume(ku, o.n, o.rank, -1);
+        if (r != ORACLE_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            rc = r;
+        }
+        for (int64_t p = 0; p < o.V; ++p) ku[p] *= mask_at(mask, &o, b, t, p);
+    }
+    return rc;
+}
+
+/* img = A^H k:  img[b,t] = sum_c conj(S_c) .* F^H (M .* k_c).   k is overwritten (scratch). */
+int oracle_apply_AH(zc* k, const float* sens, const float* mask, const int64_t* dims,
+                    zc* img, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK) return ORACLE_ERR_ARG;
+    int rc = ORACLE_OK;
+    const int64_t units = o.B * o.C * o.T;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(dynamic, 1)
+#endif
+    for (int64_t u = 0; u < units; ++u) {
+        const int64_t t = u % o.T, c = (u / o.T) % o.C, b = u / (o.T * o.C);
+        const float* ss = sens_ptr(sens, &o, b, c, t);
+        zc* ku = k + u * o.V;
+        for (int64_t p = 0; p < o.V; ++p) ku[p] *= mask_at(mask, &o, b, t, p);
+        const int r = fft_centered_volume(ku, o.n, o.rank, +1);
+        if (r != ORACLE_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            rc = r;
+        }
+        for (int64_t p = 0; p < o.V; ++p) {
+            const zc sv = (double)ss[2 * p] + I * (double)ss[2 * p + 1];
+            ku[p] = conj(sv) * ku[p];
+        }
+    }
+    /* coil sum in coil order (fixed order: result independent of the thread count) */
+    for (int64_t b = 0; b < o.B; ++b)
+        for (int64_t t = 0; t < o.T; ++t) {
+            zc* dst = img + (b * o.T + t) * o.V;
+            for (int64_t p = 0; p < o.V; ++p) dst[p] = 0.0;
+            for (int64_t c = 0; c < o.C; ++c) {
+                const zc* src = k + ((b * o.C + c) * o.T + t) * o.V;
+                for (int64_t p = 0; p < o.V; ++p) dst[p] += src[p];
+            }
+        }
+    return rc;
+}
+
+/* Eq. 3 with eta = 2t:   out = x - eta * A^H (A x - y).
+ * y == NULL evaluates the vector-Jacobian product  out = x - eta * A^H A x  (x is then the
+ * incoming cotangent).  Steps, in the order of the definition:
+ *   1. c_c = S_c .* x          2. k_c = F c_c            3. r_c = M .* (M .* k_c - y_c)
+ *   4. a = sum_c conj(S_c) .* F^H r_c                    5. out = x - eta a
+ */
+int oracle_dc(const float* x, const float* y, const float* sens, const float* mask, double eta,
+              const int64_t* dims, zc* out, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK) return ORACLE_ERR_ARG;
+    if (!x || !sens || !mask || !out) return ORACLE_ERR_ARG;
+    zc* contrib = (zc*)malloc(sizeof(zc) * (size_t)(o.C * o.V));
+    if (!contrib) return ORACLE_ERR_MEM;
+    int rc = ORACLE_OK;
+    if (nthreads < 1) nthreads = 1;
+    for (int64_t b = 0; b < o.B; ++b)
+        for (int64_t t = 0; t < o.T; ++t) {
+            const float* xs = x + 2 * (b * o.T + t) * o.V;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(nthreads) schedule(dynamic, 1)
+#endif
+            for (int64_t c = 0; c < o.C; ++c) {
+                const float* ss = sens_ptr(sens, &o, b, c, t);
+                zc* w = contrib + c * o.V;
+                /* 1 */
+                for (int64_t p = 0; p < o.V; ++p) {
+                    const zc xv = (double)xs[2 * p] + I * (double)xs[2 * p + 1];
+                    const zc sv = (double)ss[2 * p] + I * (double)ss[2 * p + 1];
+                    w[p] = sv * xv;
+                }
+                /* 2 */
+                int r = fft_centered_volume(w, o.n, o.rank, -1);
+                /* 3 */
+                const float* ys = y ? y + 2 * ((b * o.C + c) * o.T + t) * o.V : NULL;
+                for (int64_t p = 0; p < o.V; ++p) {
+                    const double m = mask_at(mask, &o, b, t, p);
+                    zc res = m * w[p];
+                    if (ys) res -= (double)ys[2 * p] + I * (double)ys[2 * p + 1];
+                    w[p] = m * res;
+                }
+                /* 4 (per coil) */
+                if (r == ORACLE_OK) r = fft_centered_volume(w, o.n, o.rank, +1);
+                for (int64_t p = 0; p < o.V; ++p) {
+                    const zc sv = (double)ss[2 * p] + I * (double)ss[2 * p + 1];
+                    w[p] = conj(sv) * w[p];
+                }
+                if (r != ORACLE_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+                    rc = r;
+                }
+            }
+            /* 4 (coil sum, fixed order) and 5 */
+            zc* dst = out + (b * o.T + t) * o.V;
+            for (int64_t p = 0; p < o.V; ++p) {
+                zc a = 0.0;
+                for (int64_t c = 0; c < o.C; ++c) a += contrib[c * o.V + p];
+                const zc xv = (double)xs[2 * p] + I * (double)xs[2 * p + 1];
+                dst[p] = xv - eta * a;
+            }
+        }
+    free(contrib);
+    return rc;
+}
+
+int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

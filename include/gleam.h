@@ -1,0 +1,129 @@
+/*
+ * gleam.h — C ABI of the B200 (sm_100a) multi-coil SENSE data-consistency library.
+ *
+ * The library computes the data-consistency step of the unrolled proximal-gradient network of
+ * GLEAM (arXiv 2207.08393) and its vector-Jacobian product:
+ *
+ *     sensing model (Eq. 1)            y = Omega F S x + eps
+ *     forward operator (after Eq. 2)   A = Omega F S,  A^H its Hermitian transpose
+ *     data consistency (Eq. 3)         DC(x) = x - 2t A^H (A x - y)            eta := 2t
+ *     Jacobian of Eq. 3                J = I - eta A^H A   (Hermitian for real eta)
+ *
+ * S multiplies the image by each coil's sensitivity map, F is the centred orthonormal DFT over the
+ * trailing fft_rank spatial axes (centre index floor(N/2) in both domains, kernel
+ * exp(-2 pi i (k-o)(n-o)/N) / sqrt(N)), Omega multiplies k-space by a real sampling weight
+ * (normally 0/1).  Omega is applied once in A and once more in A^H, as the definition says:
+ * r_c = M .* (M .* F(S_c .* x) - y_c).
+ *
+ * Data layout: every array is contiguous, row-major, last index fastest.  complex64 means
+ * interleaved {float re, float im}.
+ *     x, out, grad_out, grad_in : (B, T, n0, n1, n2)           complex64
+ *     y                         : (B, C, T, n0, n1, n2)        complex64
+ *     sens                      : (B, C, n0, n1, n2) or (B, C, T, n0, n1, n2)   complex64
+ *     mask                      : see mask_kind                 float32
+ * B batch, C coils, T frames (never transformed), n0 = 1 when fft_rank == 2.
+ *
+ * Ownership: all data pointers are DEVICE pointers owned by the caller.  The library neither
+ * allocates nor frees device memory and keeps no pointer after the call returns.  Work is
+ * enqueued on dims->stream and the call returns without synchronising; the buffers (including the
+ * workspace) must stay valid and untouched until that work has completed.
+ *
+ * Errors: every function returns GLEAM_OK (0) or a negative GLEAM_ERR_* code.  Argument checks
+ * run on the host before anything is enqueued; a call that returns an argument error has launched
+ * nothing.  GLEAM_ERR_CUDA reports a failed launch; kernels enqueued before it may still run.
+ * Unsupported transform lengths are reported (GLEAM_ERR_UNSUPPORTED_SIZE), never emulated on the
+ * CPU.  Results are deterministic: the same inputs give bit-identical outputs on every call.
+ */
+#ifndef GLEAM_H_
+#define GLEAM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define GLEAM_API __attribute__((visibility("default")))
+#else
+#define GLEAM_API
+#endif
+
+#define GLEAM_VERSION 1
+#define GLEAM_DIMS_VERSION 1
+
+enum {
+    GLEAM_OK = 0,
+    GLEAM_ERR_NULL_POINTER = -1,
+    GLEAM_ERR_BAD_DIMS = -2,
+    GLEAM_ERR_UNSUPPORTED_SIZE = -3,
+    GLEAM_ERR_NOT_DEVICE_POINTER = -4,
+    GLEAM_ERR_WORKSPACE_TOO_SMALL = -5,
+    GLEAM_ERR_ALIAS = -6,
+    GLEAM_ERR_CUDA = -7,
+    GLEAM_ERR_UNIMPLEMENTED = -8,
+    GLEAM_ERR_TIMEOUT = -9
+};
+
+enum {
+    GLEAM_MASK_FULL = 0,             /* mask is (B, T, n0, n1, n2) */
+    GLEAM_MASK_READOUT_INVARIANT = 1 /* mask does not depend on the readout index:
+                                        fft_rank 2 -> (B, T, n2)      (readout axis n1)
+                                        fft_rank 3 -> (B, T, n1, n2)  (readout axis n0) */
+};
+
+typedef struct {
+    int32_t struct_version;  /* GLEAM_DIMS_VERSION */
+    int32_t batch;           /* B >= 1 */
+    int32_t coils;           /* C >= 1 */
+    int32_t frames;          /* T >= 1; the frame axis is not transformed */
+    int32_t fft_rank;        /* 2 or 3 */
+    int32_t n[3];            /* n0, n1, n2 (slowest to fastest); n0 = 1 when fft_rank == 2 */
+    int32_t sens_has_frames; /* 0: sens is (B,C,n0,n1,n2); 1: (B,C,T,n0,n1,n2) */
+    int32_t mask_kind;       /* GLEAM_MASK_* ; the mask is broadcast over coils */
+    void* stream;            /* cudaStream_t; NULL = the legacy default stream */
+    void* workspace;         /* device scratch of at least gleam_dc_workspace_size() bytes,
+                                256-byte aligned; its contents are undefined afterwards */
+    uint64_t workspace_bytes;
+} gleam_dims;
+
+/*
+ * Data-consistency step, Eq. 3:   out = x - eta * A^H (A x - y).
+ *   x, y, sens, mask, out : device pointers, layouts above.  out may be exactly x (in place);
+ *   any other overlap between an output or the workspace and another argument is
+ *   GLEAM_ERR_ALIAS.  y may hold anything where the mask is zero: those samples are not read.
+ *   eta : real step size (2t in the paper's notation).
+ */
+GLEAM_API int gleam_dc_forward(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                     void* out, const gleam_dims* dims);
+
+/*
+ * Vector-Jacobian product of Eq. 3 with respect to x:   grad_in = grad_out - eta * A^H A grad_out
+ * (J^H g with J = I - eta A^H A; the conjugate-Wirtinger convention for complex tensors).
+ * grad_in may be exactly grad_out.
+ */
+GLEAM_API int gleam_dc_vjp(const void* grad_out, const void* sens, const float* mask, float eta,
+                 void* grad_in, const gleam_dims* dims);
+
+/*
+ * Scratch bytes that gleam_dc_forward / gleam_dc_vjp need for these dims (the larger of the two).
+ * Reads only the shape fields of dims; stream and workspace are ignored.
+ */
+GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes);
+
+/*
+ * GLEAM_OK if a transform of this length is supported along an axis (even lengths whose plan is
+ * compiled in), GLEAM_ERR_UNSUPPORTED_SIZE otherwise.
+ */
+GLEAM_API int gleam_dc_length_supported(int32_t n);
+
+/* Static, human-readable text for a status code. */
+GLEAM_API const char* gleam_status_string(int status);
+
+/* GLEAM_VERSION of the loaded library. */
+GLEAM_API int gleam_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GLEAM_H_ */

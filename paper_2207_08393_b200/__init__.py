@@ -3,5 +3,8 @@ vector-Jacobian product.  The arithmetic lives in the CUDA library ``libgleam_dc
 ``include/gleam.h``); this package is the argument-marshalling binding plus the seeded synthetic
 workload generators."""
 from . import workloads  # noqa: F401
-
-__all__ = ["workloads"]
+from .binding import (  # noqa: F401
+    DataConsistency, GleamError, GLEAM_MASK_FULL, GLEAM_MASK_READOUT_INVARIANT, gleam_dc_forward,
+    gleam_dc_length_supported, gleam_dc_vjp, gleam_dc_workspace_size, gleam_dims, gleam_status_string,
+    gleam_version, load_library, make_dims,
+)

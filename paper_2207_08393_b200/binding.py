@@ -1,0 +1,179 @@
+"""ctypes binding of ``libgleam_dc.so`` (C ABI: include/gleam.h).
+
+Argument marshalling only: every arithmetic step runs in the CUDA library.  The functions carry
+the same names and argument order as the C entry points and accept torch CUDA tensors (or raw
+integer device addresses).  There is no CPU fallback: if the shared library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libgleam_dc.so")
+
+GLEAM_OK = 0
+GLEAM_ERR_NULL_POINTER = -1
+GLEAM_ERR_BAD_DIMS = -2
+GLEAM_ERR_UNSUPPORTED_SIZE = -3
+GLEAM_ERR_NOT_DEVICE_POINTER = -4
+GLEAM_ERR_WORKSPACE_TOO_SMALL = -5
+GLEAM_ERR_ALIAS = -6
+GLEAM_ERR_CUDA = -7
+GLEAM_ERR_UNIMPLEMENTED = -8
+GLEAM_ERR_TIMEOUT = -9
+
+GLEAM_MASK_FULL = 0
+GLEAM_MASK_READOUT_INVARIANT = 1
+
+EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam_dc_length_supported",
+           "gleam_status_string", "gleam_version"]
+
+
+class gleam_dims(ctypes.Structure):
+    _fields_ = [
+        ("struct_version", ctypes.c_int32),
+        ("batch", ctypes.c_int32),
+        ("coils", ctypes.c_int32),
+        ("frames", ctypes.c_int32),
+        ("fft_rank", ctypes.c_int32),
+        ("n", ctypes.c_int32 * 3),
+        ("sens_has_frames", ctypes.c_int32),
+        ("mask_kind", ctypes.c_int32),
+        ("stream", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_uint64),
+    ]
+
+
+class GleamError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__("gleam status %d: %s" % (status, text))
+        self.status = status
+
+
+_lib = None
+
+
+def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(path):
+            raise RuntimeError(
+                "%s is missing: build it with `python -m paper_2207_08393_b200._build` "
+                "(there is no CPU fallback)" % path)
+        lib = ctypes.CDLL(path)
+        vp, f32, i32 = ctypes.c_void_p, ctypes.c_float, ctypes.c_int
+        dp = ctypes.POINTER(gleam_dims)
+        lib.gleam_dc_forward.argtypes = [vp, vp, vp, vp, f32, vp, dp]
+        lib.gleam_dc_forward.restype = i32
+        lib.gleam_dc_vjp.argtypes = [vp, vp, vp, f32, vp, dp]
+        lib.gleam_dc_vjp.restype = i32
+        lib.gleam_dc_workspace_size.argtypes = [dp, ctypes.POINTER(ctypes.c_uint64)]
+        lib.gleam_dc_workspace_size.restype = i32
+        lib.gleam_dc_length_supported.argtypes = [ctypes.c_int32]
+        lib.gleam_dc_length_supported.restype = i32
+        lib.gleam_status_string.argtypes = [i32]
+        lib.gleam_status_string.restype = ctypes.c_char_p
+        lib.gleam_version.argtypes = []
+        lib.gleam_version.restype = i32
+        _lib = lib
+    return _lib
+
+
+def gleam_status_string(status: int) -> str:
+    return load_library().gleam_status_string(int(status)).decode()
+
+
+def gleam_version() -> int:
+    return int(load_library().gleam_version())
+
+
+def gleam_dc_length_supported(n: int) -> bool:
+    return load_library().gleam_dc_length_supported(int(n)) == GLEAM_OK
+
+
+def _addr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return int(t.data_ptr())
+
+
+def _check(status: int):
+    if status != GLEAM_OK:
+        raise GleamError(status, gleam_status_string(status))
+
+
+def make_dims(batch, coils, frames, fft_rank, n, sens_has_frames=0, mask_kind=GLEAM_MASK_READOUT_INVARIANT,
+              stream=None, workspace=None, workspace_bytes=0) -> gleam_dims:
+    """Fills a ``gleam_dims``.  ``stream`` is a torch.cuda.Stream, a raw handle or None (legacy
+    default stream); ``workspace`` a torch uint8 CUDA tensor or a raw address."""
+    d = gleam_dims()
+    d.struct_version = 1
+    d.batch, d.coils, d.frames, d.fft_rank = int(batch), int(coils), int(frames), int(fft_rank)
+    d.n[0], d.n[1], d.n[2] = int(n[0]), int(n[1]), int(n[2])
+    d.sens_has_frames, d.mask_kind = int(sens_has_frames), int(mask_kind)
+    if stream is not None and not isinstance(stream, int):
+        stream = stream.cuda_stream
+    d.stream = stream or None
+    if workspace is not None and not isinstance(workspace, int):
+        workspace_bytes = workspace.numel() * workspace.element_size()
+        workspace = workspace.data_ptr()
+    d.workspace = workspace or None
+    d.workspace_bytes = int(workspace_bytes)
+    return d
+
+
+def gleam_dc_workspace_size(dims: gleam_dims) -> int:
+    out = ctypes.c_uint64(0)
+    _check(load_library().gleam_dc_workspace_size(ctypes.byref(dims), ctypes.byref(out)))
+    return int(out.value)
+
+
+def gleam_dc_forward(x, y, sens, mask, eta, out, dims: gleam_dims) -> None:
+    """out = x - eta A^H (A x - y)  (Eq. 3, eta = 2t).  Enqueues on dims.stream and returns."""
+    _check(load_library().gleam_dc_forward(_addr(x), _addr(y), _addr(sens), _addr(mask), float(eta), _addr(out),
+                                            ctypes.byref(dims)))
+
+
+def gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, dims: gleam_dims) -> None:
+    """grad_in = grad_out - eta A^H A grad_out  (VJP of Eq. 3 with respect to x)."""
+    _check(load_library().gleam_dc_vjp(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
+                                        ctypes.byref(dims)))
+
+
+class DataConsistency:
+    """Convenience holder: dims + a workspace tensor for one problem shape on the current device
+    and stream.  ``forward`` / ``vjp`` allocate their output unless one is passed."""
+
+    def __init__(self, batch, coils, frames, fft_rank, n, sens_has_frames=0,
+                 mask_kind=GLEAM_MASK_READOUT_INVARIANT, stream=None):
+        import torch
+        self._torch = torch
+        probe = make_dims(batch, coils, frames, fft_rank, n, sens_has_frames, mask_kind)
+        nbytes = gleam_dc_workspace_size(probe)
+        self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        self.shape = (batch, frames) + tuple(int(v) for v in n)
+        self._args = (batch, coils, frames, fft_rank, n, sens_has_frames, mask_kind)
+        self.stream = stream
+
+    def dims(self) -> gleam_dims:
+        torch = self._torch
+        st = self.stream if self.stream is not None else torch.cuda.current_stream()
+        return make_dims(*self._args, stream=st, workspace=self.workspace)
+
+    def forward(self, x, y, sens, mask, eta, out=None):
+        if out is None:
+            out = self._torch.empty_like(x)
+        gleam_dc_forward(x, y, sens, mask, eta, out, self.dims())
+        return out
+
+    def vjp(self, grad_out, sens, mask, eta, grad_in=None):
+        if grad_in is None:
+            grad_in = self._torch.empty_like(grad_out)
+        gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, self.dims())
+        return grad_in

@@ -1,0 +1,311 @@
+// Kernels of the data-consistency step  out = x - eta * A^H (A x - y),  A = Omega F S  (Eq. 3 of
+// the GLEAM paper with eta = 2t; sensing model Eq. 1) and of its vector-Jacobian product.
+//
+// All transforms inside the kernels are raw DFTs.  Centring and orthonormal scaling of F are moved
+// into the k-space tables: with the shift sh(k) = (k + N/2) mod N per transformed axis,
+//     A^H A   = S^H  Fraw^H  diag( M[sh(k)]^2 / N )  Fraw  S
+//     A^H y   = S^H  Fraw^H  ( g (-1)^{sh(k)} M[sh(k)] y[sh(k)] / sqrt(N) ),   g = prod (-1)^{N_a/2}
+// (even extents only).
+//
+// ROW kernels transform the contiguous axis n2 and carry the image-side work (sensitivity
+// multiply on the way in, conjugate-sensitivity coil sum in registers on the way out).
+// COL kernels transform a strided axis in place on a workspace, or turn y into the table z.
+#pragma once
+#include "fft_line.cuh"
+#include <stdint.h>
+
+namespace gleam {
+
+enum RowMode { ROW_FUSED = 0, ROW_FWD = 1, ROW_INV = 2 };
+enum ColMode { COL_Z = 0, COL_MID_SEP = 1, COL_MID_FULL = 2, COL_FWD = 3, COL_INV = 4 };
+
+struct RowArgs {
+    const cf* x;        // image-domain input (B,T,n0,n1,n2)
+    const cf* sens;     // (B,C,[T],n0,n1,n2)
+    cf* out;            // (B,T,n0,n1,n2)
+    const float* m2;    // ROW_FUSED: (B,T,n2) shifted mask^2 / n2
+    const cf* z;        // ROW_FUSED: (B,C,T,n1,n2) shifted, signed, masked R^H y; may be null
+    cf* W;              // workspace (unit, rpb, n2)
+    float eta;
+    int C, T, Ts;       // coils, frames, sens frames (T or 1)
+    int rpb;            // rows of this launch per (b,t)
+    int row0;           // first row of this launch inside the full image rows
+    int RPB;            // rows of a full image (n0*n1)
+    long long nrows;    // B*T*rpb
+};
+
+struct ColArgs {
+    cf* W;              // in-place data (COL_MID_*, COL_FWD, COL_INV)
+    const cf* y;        // COL_Z input / COL_MID_FULL measurements (B,C,T,V)
+    cf* z;              // COL_Z output
+    const cf* zin;      // COL_MID_SEP: z table (unit, n0, n1, n2)
+    const float* mask;  // COL_Z: readout-invariant mask; COL_MID_FULL: full mask (B,T,V)
+    const float* m2;    // COL_MID_SEP: (B,T,n1,n2) shifted mask^2 / (n1 n2)
+    int es;             // element stride of the transformed axis = lines per outer index
+    long long nouter;   // outer indices
+    int C, T;
+    int rank, n0, n1, n2;
+    int G, i0_start;    // COL_MID_SEP chunk: slabs in the chunk, first slab
+    float scale;        // COL_Z: g_ro g_pe / sqrt(N_ro N_pe);  COL_MID_FULL: g / sqrt(Ntot)
+    float scale2;       // COL_MID_FULL: 1 / Ntot
+};
+
+__device__ __forceinline__ int shift_half(int k, int n) { int h = n >> 1; return k >= n - h ? k - (n - h) : k + h; }
+
+// --------------------------------------------------------------------------------------------
+// ROW kernel: L contiguous lines per block, all coils looped inside the block.
+// --------------------------------------------------------------------------------------------
+template <class P, int L, int MODE>
+__global__ void __launch_bounds__(LineFFT<P, false, L>::THREADS)
+row_kernel(const RowArgs a) {
+    using E = LineFFT<P, false, L>;
+    constexpr int N = P::N, R0 = P::R0, RL = P::RL;
+    extern __shared__ float2 smem[];
+    const typename E::Ids d = E::ids(threadIdx.x);
+    typename E::Tw tw;
+    E::make_tw(d, tw);
+
+    // first-stage identity of this thread
+    const long long r0 = (long long)blockIdx.x * L + d.l0;
+    const bool act0 = d.a0 && r0 < a.nrows;
+    const long long bt0 = act0 ? r0 / a.rpb : 0;
+    const int ri0 = act0 ? (int)(r0 % a.rpb) : 0;
+    const int b0 = (int)(bt0 / a.T), t0 = (int)(bt0 % a.T);
+    // last-stage identity
+    const long long rL = (long long)blockIdx.x * L + d.lL;
+    const bool actL = d.aL && rL < a.nrows;
+    const long long btL = actL ? rL / a.rpb : 0;
+    const int riL = actL ? (int)(rL % a.rpb) : 0;
+    const int bL = (int)(btL / a.T), tL = (int)(btL % a.T);
+
+    const long long x_off = ((long long)bt0 * a.RPB + a.row0 + ri0) * N;
+    cf xv[R0], acc[R0];
+    if (MODE != ROW_FWD) {
+#pragma unroll
+        for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
+    }
+    if (act0) {
+#pragma unroll
+        for (int m = 0; m < R0; ++m) xv[m] = a.x[x_off + d.j0 + P::BF0 * m];
+    }
+    float m2v[RL];
+    if (MODE == ROW_FUSED) {
+        if (actL) {
+#pragma unroll
+            for (int k = 0; k < RL; ++k) m2v[k] = a.m2[btL * N + d.jL + P::BFL * k];
+        }
+    }
+
+    for (int c = 0; c < a.C; ++c) {
+        const long long s_off = (((long long)(b0 * a.C + c) * a.Ts + (a.Ts > 1 ? t0 : 0)) * a.RPB + a.row0 + ri0) * N;
+        cf v[R0], u[RL];
+        if (MODE != ROW_INV) {
+            if (act0) {
+#pragma unroll
+                for (int m = 0; m < R0; ++m) v[m] = cmul(a.sens[s_off + d.j0 + P::BF0 * m], xv[m]);
+            } else {
+#pragma unroll
+                for (int m = 0; m < R0; ++m) v[m] = make_float2(0.f, 0.f);
+            }
+            E::forward(v, u, tw, d, smem);
+        }
+        if (MODE == ROW_FUSED) {
+            if (actL) {
+                if (a.z) {
+                    const long long z_off = (((long long)(bL * a.C + c) * a.T + tL) * a.RPB + a.row0 + riL) * N;
+#pragma unroll
+                    for (int k = 0; k < RL; ++k) {
+                        const cf zz = a.z[z_off + d.jL + P::BFL * k];
+                        u[k] = make_float2(fmaf(m2v[k], u[k].x, -zz.x), fmaf(m2v[k], u[k].y, -zz.y));
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], m2v[k]);
+                }
+            }
+        } else if (MODE == ROW_FWD) {
+            if (actL) {
+                const long long w_off = (((long long)(bL * a.C + c) * a.T + tL) * a.rpb + riL) * N;
+#pragma unroll
+                for (int k = 0; k < RL; ++k) a.W[w_off + d.jL + P::BFL * k] = u[k];
+            }
+        } else {  // ROW_INV
+            if (actL) {
+                const long long w_off = (((long long)(bL * a.C + c) * a.T + tL) * a.rpb + riL) * N;
+#pragma unroll
+                for (int k = 0; k < RL; ++k) u[k] = a.W[w_off + d.jL + P::BFL * k];
+            }
+        }
+        if (MODE != ROW_FWD) {
+            E::inverse(u, v, tw, d, smem);
+            if (act0) {
+#pragma unroll
+                for (int m = 0; m < R0; ++m) {
+                    const cf s = a.sens[s_off + d.j0 + P::BF0 * m];
+                    // acc += conj(s) * v
+                    acc[m].x = fmaf(s.x, v[m].x, fmaf(s.y, v[m].y, acc[m].x));
+                    acc[m].y = fmaf(s.x, v[m].y, fmaf(-s.y, v[m].x, acc[m].y));
+                }
+            }
+        }
+    }
+    if (MODE != ROW_FWD) {
+        if (act0) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m)
+                a.out[x_off + d.j0 + P::BF0 * m] =
+                    make_float2(fmaf(-a.eta, acc[m].x, xv[m].x), fmaf(-a.eta, acc[m].y, xv[m].y));
+        }
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// COL kernel: L neighbouring strided lines per block.
+// --------------------------------------------------------------------------------------------
+template <class P, int L, int MODE>
+__global__ void __launch_bounds__(LineFFT<P, true, L>::THREADS)
+col_kernel(const ColArgs a) {
+    using E = LineFFT<P, true, L>;
+    constexpr int N = P::N, R0 = P::R0, RL = P::RL;
+    extern __shared__ float2 smem[];
+    const typename E::Ids d = E::ids(threadIdx.x);
+    typename E::Tw tw;
+    E::make_tw(d, tw);
+
+    const int tiles = (a.es + L - 1) / L;
+    const long long o = blockIdx.x / tiles;           // outer index
+    const int i_base = (int)(blockIdx.x % tiles) * L;
+    // COL mode: every stage sees the same line index l = tid % L
+    const int i = i_base + d.l0;
+    const bool line_ok = i < a.es;
+    const bool act0 = d.a0 && line_ok, actL = d.aL && line_ok;
+    const long long base = o * (long long)N * a.es + i;
+
+    cf v[R0], u[RL];
+
+    if (MODE == COL_Z) {
+        // z = (g/sqrt(N_ro N_pe)) (-1)^{n_ro} (-1)^{p} M[p] * Rraw^H( (-1)^{k_ro} y ),  stored at sh(p)
+        // outer o = unit (b,c,t); inner i = phase-encode position p (flat over n1,n2 for rank 3)
+        const int t = (int)(o % a.T);
+        const int b = (int)(o / ((long long)a.C * a.T));
+        float mv = 0.f; int dest = 0, psign = 0;
+        if (line_ok) {
+            const long long pe = a.es;
+            mv = a.mask[((long long)b * a.T + t) * pe + i];
+            if (a.rank == 2) { dest = shift_half(i, a.n2); psign = i & 1; }
+            else {
+                const int i1 = i / a.n2, i2 = i % a.n2;
+                dest = shift_half(i1, a.n1) * a.n2 + shift_half(i2, a.n2);
+                psign = (i1 + i2) & 1;
+            }
+        }
+        if (actL) {
+#pragma unroll
+            for (int k = 0; k < RL; ++k) {
+                const int kk = d.jL + P::BFL * k;
+                cf yv = (mv != 0.f) ? a.y[base + (long long)kk * a.es] : make_float2(0.f, 0.f);
+                u[k] = (kk & 1) ? make_float2(-yv.x, -yv.y) : yv;
+            }
+        }
+        E::inverse(u, v, tw, d, smem);
+        if (act0) {
+            const float f = (psign ? -a.scale : a.scale) * mv;
+#pragma unroll
+            for (int m = 0; m < R0; ++m) {
+                const int n = d.j0 + P::BF0 * m;
+                const float ff = (n & 1) ? -f : f;
+                a.z[o * (long long)N * a.es + (long long)n * a.es + dest] = cscale(v[m], ff);
+            }
+        }
+        return;
+    }
+
+    if (MODE == COL_INV) {
+        if (actL) {
+#pragma unroll
+            for (int k = 0; k < RL; ++k) u[k] = a.W[base + (long long)(d.jL + P::BFL * k) * a.es];
+        }
+    } else {
+        if (act0) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) v[m] = a.W[base + (long long)(d.j0 + P::BF0 * m) * a.es];
+        } else {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) v[m] = make_float2(0.f, 0.f);
+        }
+        E::forward(v, u, tw, d, smem);
+    }
+
+    if (MODE == COL_FWD) {
+        if (actL) {
+#pragma unroll
+            for (int k = 0; k < RL; ++k) a.W[base + (long long)(d.jL + P::BFL * k) * a.es] = u[k];
+        }
+        return;
+    }
+
+    if (MODE == COL_MID_SEP) {
+        // W chunk (unit, G, n1, n2), axis n1, es = n2.  o = unit*G + gi
+        if (actL) {
+            const long long unit = o / a.G;
+            const int gi = (int)(o % a.G);
+            const int t = (int)(unit % a.T);
+            const int b = (int)(unit / ((long long)a.C * a.T));
+            const long long pe = (long long)a.n1 * a.n2;
+            const float* m2 = a.m2 + ((long long)b * a.T + t) * pe + i;
+            const cf* zz = a.zin ? a.zin + (unit * a.n0 + a.i0_start + gi) * pe + i : nullptr;
+#pragma unroll
+            for (int k = 0; k < RL; ++k) {
+                const long long kk = (long long)(d.jL + P::BFL * k) * a.n2;
+                const float w = m2[kk];
+                if (zz) {
+                    const cf q = zz[kk];
+                    u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
+                } else {
+                    u[k] = cscale(u[k], w);
+                }
+            }
+        }
+    } else if (MODE == COL_MID_FULL) {
+        // W (unit, V); the transformed axis is the readout axis (n1 for rank 2, n0 for rank 3);
+        // mask and y are read at the half-shifted k-space position on every transformed axis.
+        if (actL) {
+            const long long unit = o;
+            const int t = (int)(unit % a.T);
+            const int b = (int)(unit / ((long long)a.C * a.T));
+            const long long V = (long long)a.n0 * a.n1 * a.n2;
+            const float* mk = a.mask + ((long long)b * a.T + t) * V;
+            const cf* yy = a.y ? a.y + unit * V : nullptr;
+#pragma unroll
+            for (int k = 0; k < RL; ++k) {
+                const int kk = d.jL + P::BFL * k;
+                long long ps; int par;
+                if (a.rank == 2) {
+                    const int s1 = shift_half(kk, a.n1), s2 = shift_half(i, a.n2);
+                    ps = (long long)s1 * a.n2 + s2; par = (s1 + s2) & 1;
+                } else {
+                    const int i1 = i / a.n2, i2 = i % a.n2;
+                    const int s0 = shift_half(kk, a.n0), s1 = shift_half(i1, a.n1), s2 = shift_half(i2, a.n2);
+                    ps = ((long long)s0 * a.n1 + s1) * a.n2 + s2; par = (s0 + s1 + s2) & 1;
+                }
+                const float mv = mk[ps];
+                const float w = mv * mv * a.scale2;
+                if (yy) {
+                    const cf q = yy[ps];
+                    const float f = (par ? -a.scale : a.scale) * mv;
+                    u[k] = make_float2(fmaf(w, u[k].x, -f * q.x), fmaf(w, u[k].y, -f * q.y));
+                } else {
+                    u[k] = cscale(u[k], w);
+                }
+            }
+        }
+    }
+
+    E::inverse(u, v, tw, d, smem);
+    if (act0) {
+#pragma unroll
+        for (int m = 0; m < R0; ++m) a.W[base + (long long)(d.j0 + P::BF0 * m) * a.es] = v[m];
+    }
+}
+
+}  // namespace gleam

@@ -1,0 +1,280 @@
+// Host side of the C ABI declared in include/gleam.h: argument validation, workspace layout and
+// the sequence of kernel launches for each problem class.
+//
+//   readout-invariant mask, fft_rank 2 :  [z = R^H y table]  ->  fused row kernel (one pass)
+//   readout-invariant mask, fft_rank 3 :  [z table]  ->  per chunk of readout slabs:
+//                                         rows forward -> columns (mask, residual) -> rows inverse
+//   full mask                           :  rows forward -> strided axes -> rows inverse on a
+//                                         coil-volume workspace
+//
+// With a mask that does not depend on the readout index the readout transform commutes with the
+// mask, so A^H(Ax - y) = S^H P^H M (M P S x - R^H y) with P over the phase-encode axes and R over
+// the readout axis only; R^H y is needed at sampled positions alone.
+#include "../../include/gleam.h"
+#include "size_ops.cuh"
+
+#include <cstdlib>
+#include <cmath>
+
+namespace gleam {
+
+#define GLEAM_SIZE(N, R0, R1, R2, LR, LC) extern const SizeOps size_ops_##N;
+#include "sizes.def"
+#undef GLEAM_SIZE
+
+static const SizeOps* find_size(int n) {
+    switch (n) {
+#define GLEAM_SIZE(N, R0, R1, R2, LR, LC) case N: return &size_ops_##N;
+#include "sizes.def"
+#undef GLEAM_SIZE
+        default: return nullptr;
+    }
+}
+
+// shifted mask^2 * scale table for the separable paths:  m2[bt][k] = M[bt][sh(k)]^2 * scale
+__global__ void prep_m2_kernel(const float* __restrict__ mask, float* __restrict__ m2, long long nbt,
+                               int n1, int n2, int rank, float scale) {
+    const long long pe = (rank == 2) ? n2 : (long long)n1 * n2;
+    const long long tot = nbt * pe;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < tot;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const long long bt = idx / pe;
+        const int p = (int)(idx % pe);
+        int src;
+        if (rank == 2) src = shift_half(p, n2);
+        else src = shift_half(p / n2, n1) * n2 + shift_half(p % n2, n2);
+        const float mv = mask[bt * pe + src];
+        m2[idx] = mv * mv * scale;
+    }
+}
+
+static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    // geometry
+    int B, C, T, Ts, rank, n0, n1, n2;
+    long long V, units, images;
+    bool separable;
+    // workspace (byte offsets)
+    uint64_t off_m2, off_z, off_W, total;
+    int G;  // readout slabs per chunk (rank 3 separable)
+};
+
+static const uint64_t CHUNK_TARGET_BYTES = 48ull << 20;   // keep the chunk workspace inside L2
+
+static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
+    if (d->struct_version != GLEAM_DIMS_VERSION) return GLEAM_ERR_BAD_DIMS;
+    if (d->batch < 1 || d->coils < 1 || d->frames < 1) return GLEAM_ERR_BAD_DIMS;
+    if (d->fft_rank != 2 && d->fft_rank != 3) return GLEAM_ERR_BAD_DIMS;
+    if (d->n[0] < 1 || d->n[1] < 1 || d->n[2] < 1) return GLEAM_ERR_BAD_DIMS;
+    if (d->fft_rank == 2 && d->n[0] != 1) return GLEAM_ERR_BAD_DIMS;
+    if (d->sens_has_frames != 0 && d->sens_has_frames != 1) return GLEAM_ERR_BAD_DIMS;
+    if (d->mask_kind != GLEAM_MASK_FULL && d->mask_kind != GLEAM_MASK_READOUT_INVARIANT) return GLEAM_ERR_BAD_DIMS;
+    for (int a = 3 - d->fft_rank; a < 3; ++a)
+        if (!find_size(d->n[a])) return GLEAM_ERR_UNSUPPORTED_SIZE;
+    L->B = d->batch; L->C = d->coils; L->T = d->frames; L->Ts = d->sens_has_frames ? d->frames : 1;
+    L->rank = d->fft_rank; L->n0 = d->n[0]; L->n1 = d->n[1]; L->n2 = d->n[2];
+    L->V = (long long)L->n0 * L->n1 * L->n2;
+    L->images = (long long)L->B * L->T;
+    L->units = L->images * L->C;
+    if (L->V > (1ll << 40) || L->units * L->V > (1ll << 46)) return GLEAM_ERR_BAD_DIMS;
+    L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
+    uint64_t off = 0;
+    L->off_m2 = L->off_z = L->off_W = 0; L->G = 0;
+    if (L->separable) {
+        const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
+        L->off_m2 = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(float), 256);
+        if (with_y) { L->off_z = off; off = align_up(off + (uint64_t)L->units * L->V * sizeof(cf), 256); }
+        if (L->rank == 3) {
+            const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
+            long long G = (long long)(CHUNK_TARGET_BYTES / slab);
+            if (G < 1) G = 1;
+            if (G > L->n0) G = L->n0;
+            L->G = (int)G;
+            L->off_W = off; off = align_up(off + slab * (uint64_t)G, 256);
+        }
+    } else {
+        L->off_W = off; off = align_up(off + (uint64_t)L->units * L->V * sizeof(cf), 256);
+    }
+    L->total = off;
+    return GLEAM_OK;
+}
+
+static bool check_pointers_enabled() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("GLEAM_SKIP_POINTER_CHECK"); v = (e && e[0] == '1') ? 0 : 1; }
+    return v == 1;
+}
+
+static int check_device_ptr(const void* p) {
+    if (!check_pointers_enabled()) return GLEAM_OK;
+    cudaPointerAttributes at;
+    cudaError_t e = cudaPointerGetAttributes(&at, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return GLEAM_ERR_NOT_DEVICE_POINTER; }
+    if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) return GLEAM_ERR_NOT_DEVICE_POINTER;
+    return GLEAM_OK;
+}
+
+static bool overlaps(const void* a, uint64_t na, const void* b, uint64_t nb) {
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+static inline float gsign(int n) { return ((n / 2) % 2) ? -1.f : 1.f; }
+
+#define CK(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return GLEAM_ERR_CUDA; } while (0)
+
+static int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
+               const gleam_dims* d) {
+    if (!d) return GLEAM_ERR_NULL_POINTER;
+    if (!x || !sens || !mask || !out) return GLEAM_ERR_NULL_POINTER;
+    Layout L;
+    int rc = make_layout(d, y != nullptr, &L);
+    if (rc != GLEAM_OK) return rc;
+    if (L.total > 0 && !d->workspace) return GLEAM_ERR_NULL_POINTER;
+    if (d->workspace_bytes < L.total) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    if (((uintptr_t)d->workspace & 255) != 0) return GLEAM_ERR_BAD_DIMS;
+
+    const uint64_t img_b = (uint64_t)L.images * L.V * sizeof(cf);
+    const uint64_t ksp_b = (uint64_t)L.units * L.V * sizeof(cf);
+    const uint64_t sens_b = (uint64_t)L.B * L.C * L.Ts * L.V * sizeof(cf);
+    const long long pe = (L.rank == 2) ? L.n2 : (long long)L.n1 * L.n2;
+    const uint64_t mask_b = (uint64_t)L.images * (L.separable ? pe : L.V) * sizeof(float);
+    const void* ptrs[6] = {x, y, sens, mask, out, d->workspace};
+    for (int i = 0; i < 6; ++i) {
+        if (!ptrs[i]) continue;
+        if (((uintptr_t)ptrs[i] & 7) != 0) return GLEAM_ERR_BAD_DIMS;
+        rc = check_device_ptr(ptrs[i]);
+        if (rc != GLEAM_OK) return rc;
+    }
+    // aliasing: out may equal x exactly; nothing else may overlap an output or the workspace
+    if (out != x && overlaps(out, img_b, x, img_b)) return GLEAM_ERR_ALIAS;
+    if (overlaps(out, img_b, sens, sens_b) || overlaps(out, img_b, mask, mask_b)) return GLEAM_ERR_ALIAS;
+    if (y && overlaps(out, img_b, y, ksp_b)) return GLEAM_ERR_ALIAS;
+    if (L.total > 0) {
+        const void* w = d->workspace;
+        if (overlaps(w, L.total, x, img_b) || overlaps(w, L.total, out, img_b) ||
+            overlaps(w, L.total, sens, sens_b) || overlaps(w, L.total, mask, mask_b) ||
+            (y && overlaps(w, L.total, y, ksp_b)))
+            return GLEAM_ERR_ALIAS;
+    }
+
+    cudaStream_t s = (cudaStream_t)d->stream;
+    char* ws = (char*)d->workspace;
+    const SizeOps* op2 = find_size(L.n2);
+    const SizeOps* op1 = find_size(L.n1);
+    const SizeOps* op0 = (L.rank == 3) ? find_size(L.n0) : nullptr;
+
+    RowArgs ra{};
+    ra.x = (const cf*)x; ra.sens = (const cf*)sens; ra.out = (cf*)out; ra.eta = eta;
+    ra.C = L.C; ra.T = L.T; ra.Ts = L.Ts; ra.RPB = L.n0 * L.n1;
+    ColArgs ca{};
+    ca.C = L.C; ca.T = L.T; ca.rank = L.rank; ca.n0 = L.n0; ca.n1 = L.n1; ca.n2 = L.n2;
+
+    if (L.separable) {
+        float* m2 = (float*)(ws + L.off_m2);
+        cf* z = y ? (cf*)(ws + L.off_z) : nullptr;
+        {
+            const long long tot = L.images * pe;
+            const int th = 256;
+            long long bl = (tot + th - 1) / th; if (bl > 148 * 8) bl = 148 * 8;
+            prep_m2_kernel<<<(unsigned)bl, th, 0, s>>>(mask, m2, L.images, L.n1, L.n2, L.rank, 1.0f / (float)pe);
+            CK(cudaGetLastError());
+        }
+        if (y) {
+            // z table: inverse transform of y along the readout axis, at sampled positions
+            ColArgs cz = ca;
+            cz.y = (const cf*)y; cz.z = z; cz.mask = mask;
+            cz.es = (int)pe; cz.nouter = L.units;
+            const int nro = (L.rank == 2) ? L.n1 : L.n0;
+            float g = gsign(nro) * gsign(L.n2) * (L.rank == 3 ? gsign(L.n1) : 1.f);
+            cz.scale = g / sqrtf((float)nro * (float)pe);
+            CK(((L.rank == 2) ? op1 : op0)->col(COL_Z, cz, s));
+        }
+        if (L.rank == 2) {
+            ra.m2 = m2; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
+            CK(op2->row(ROW_FUSED, ra, s));
+        } else {
+            cf* W = (cf*)(ws + L.off_W);
+            for (int i0 = 0; i0 < L.n0; i0 += L.G) {
+                const int g = (L.n0 - i0 < L.G) ? (L.n0 - i0) : L.G;
+                ra.W = W; ra.rpb = g * L.n1; ra.row0 = i0 * L.n1; ra.nrows = L.images * ra.rpb;
+                CK(op2->row(ROW_FWD, ra, s));
+                ColArgs cm = ca;
+                cm.W = W; cm.m2 = m2; cm.zin = z; cm.es = L.n2; cm.nouter = L.units * g; cm.G = g; cm.i0_start = i0;
+                CK(op1->col(COL_MID_SEP, cm, s));
+                CK(op2->row(ROW_INV, ra, s));
+            }
+        }
+    } else {
+        cf* W = (cf*)(ws + L.off_W);
+        ra.W = W; ra.rpb = L.n0 * L.n1; ra.row0 = 0; ra.nrows = L.images * ra.rpb;
+        CK(op2->row(ROW_FWD, ra, s));
+        float g = gsign(L.n2) * gsign(L.n1) * (L.rank == 3 ? gsign(L.n0) : 1.f);
+        const double ntot = (L.rank == 3) ? (double)L.V : (double)L.n1 * L.n2;
+        ColArgs cm = ca;
+        cm.W = W; cm.y = (const cf*)y; cm.mask = mask;
+        cm.scale = g / (float)sqrt(ntot); cm.scale2 = (float)(1.0 / ntot);
+        if (L.rank == 2) {
+            cm.es = L.n2; cm.nouter = L.units;
+            CK(op1->col(COL_MID_FULL, cm, s));
+        } else {
+            ColArgs c1 = ca;
+            c1.W = W; c1.es = L.n2; c1.nouter = L.units * L.n0;
+            CK(op1->col(COL_FWD, c1, s));
+            cm.es = L.n1 * L.n2; cm.nouter = L.units;
+            CK(op0->col(COL_MID_FULL, cm, s));
+            CK(op1->col(COL_INV, c1, s));
+        }
+        CK(op2->row(ROW_INV, ra, s));
+    }
+    return GLEAM_OK;
+}
+
+}  // namespace gleam
+
+extern "C" {
+
+GLEAM_API int gleam_dc_forward(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                     void* out, const gleam_dims* dims) {
+    if (!y) return GLEAM_ERR_NULL_POINTER;
+    return gleam::run(x, y, sens, mask, eta, out, dims);
+}
+
+GLEAM_API int gleam_dc_vjp(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
+                 const gleam_dims* dims) {
+    return gleam::run(grad_out, nullptr, sens, mask, eta, grad_in, dims);
+}
+
+GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes) {
+    if (!dims || !bytes) return GLEAM_ERR_NULL_POINTER;
+    gleam::Layout L;
+    int rc = gleam::make_layout(dims, true, &L);
+    if (rc != GLEAM_OK) return rc;
+    *bytes = L.total;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_length_supported(int32_t n) {
+    return gleam::find_size(n) ? GLEAM_OK : GLEAM_ERR_UNSUPPORTED_SIZE;
+}
+
+GLEAM_API const char* gleam_status_string(int status) {
+    switch (status) {
+        case GLEAM_OK: return "ok";
+        case GLEAM_ERR_NULL_POINTER: return "null pointer argument";
+        case GLEAM_ERR_BAD_DIMS: return "inconsistent or misaligned dims";
+        case GLEAM_ERR_UNSUPPORTED_SIZE: return "transform length not supported";
+        case GLEAM_ERR_NOT_DEVICE_POINTER: return "argument is not a device pointer";
+        case GLEAM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case GLEAM_ERR_ALIAS: return "arguments overlap";
+        case GLEAM_ERR_CUDA: return "CUDA runtime error";
+        case GLEAM_ERR_UNIMPLEMENTED: return "not implemented";
+        case GLEAM_ERR_TIMEOUT: return "device wait timed out";
+        default: return "unknown status";
+    }
+}
+
+GLEAM_API int gleam_version(void) { return GLEAM_VERSION; }
+
+}  // extern "C"

@@ -1,0 +1,423 @@
+"""Benchmark of the SENSE data-consistency step (forward + VJP) on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload knee3d] [--impl reference]
+
+One step = one gleam_dc_forward followed by one gleam_dc_vjp on the same synthetic workload
+(all rows of the hot path: sensitivity multiply, FFT, mask + residual, inverse FFT, coil sum,
+update, and the VJP).  `value` is voxel*coils per second with every input resident in HBM;
+`e2e` is the same metric through the host-buffer C-ABI calls with pinned host inputs, the
+host->device copies and the device->host copy of the results inside the timed region.
+
+N > 1 runs N independent replicas (the path has no exchange step); the time is the max over ranks.
+`--impl reference` times the CPU oracle (as it stands) on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dc_step_fwd_plus_vjp_throughput"
+UNIT = "voxel*coils/s"
+
+# FP32 ALU peak: 148 SMs x 128 FP32 lanes x 2 flop (FMA) x SM clock
+SM_COUNT, FP32_LANES = 148, 128
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+def fp32_peak_tflops(sm_mhz):
+    return SM_COUNT * FP32_LANES * 2 * sm_mhz * 1e6 / 1e12
+
+
+# ------------------------------------------------------------------------------------------------
+# roofline bookkeeping (algorithmic bytes / flops; N log2 N counting of the transforms)
+# ------------------------------------------------------------------------------------------------
+def north_star_roofline(w, with_y):
+    """min bytes = x + S + (y) + mask + out;  flops = 2 B C T transforms x 5 N log2 N, N = points
+    per full transform."""
+    img = w.batch * w.frames * w.V * 8
+    sens = w.batch * w.coils * w.V * 8
+    ksp = w.batch * w.coils * w.frames * w.V * 8
+    pe = w.n[2] if w.fft_rank == 2 else w.n[1] * w.n[2]
+    mask = w.batch * w.frames * pe * 4
+    nbytes = 2 * img + sens + mask + (ksp if with_y else 0)
+    npts = w.V
+    flops = 2 * w.batch * w.coils * w.frames * 5 * npts * math.log2(npts)
+    return nbytes, flops
+
+
+def kernel_work(cls, w, launches_per_call):
+    """Algorithmic (bytes, flops) of ONE launch of a kernel class for workload w.
+    Per voxel*coil: see the per-kernel table in the design doc."""
+    W = w.voxel_coils / launches_per_call        # voxel*coils one launch processes
+    C = w.coils
+    l2 = math.log2
+    if cls == "row_fwd":        # read S (8) + x (8/C), write W (8)
+        return W * (16 + 8 / C), W * (5 * l2(w.n[2]) + 6)
+    if cls == "row_inv":        # read W (8) + S (8) + x (8/C), write out (8/C)
+        return W * (16 + 16 / C), W * (5 * l2(w.n[2]) + 8)
+    if cls == "col_mid_sep":    # read + write W (16), tables
+        return W * 16, W * (10 * l2(w.n[1]) + 4)
+    if cls == "row_fused":      # read S (8) [+ z (8) in the forward call, averaged] + x/out (16/C)
+        return W * (8 + 4 + 16 / C), W * (10 * l2(w.n[2]) + 20)
+    if cls == "col_z":          # read y (8), write z (8)
+        nro = w.n[1] if w.fft_rank == 2 else w.n[0]
+        return W * 16, W * (5 * l2(nro))
+    if cls == "col_mid_full":
+        nro = w.n[1] if w.fft_rank == 2 else w.n[0]
+        return W * 24, W * (10 * l2(nro) + 6)
+    if cls in ("col_fwd", "col_inv"):
+        return W * 16, W * (5 * l2(w.n[1]))
+    return 0.0, 0.0
+
+
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.strip().split(",") for r in open(self.tmp.name) if r.strip()]
+        os.unlink(self.tmp.name)
+        sm, names = [], ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in rows:
+            try:
+                sm.append(float(r[0])); out["sm_max_mhz"] = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for nme, v in zip(names, r[3:7]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(nme)
+        if sm:
+            busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
+            out["sm_mhz"] = statistics.median(busy)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def aggregate(local_ms, local_units, world, dist=None, device=None):
+    """Whole-job numbers from per-rank ones: time = max over ranks, units = sum over ranks.
+    With world == 1 no process group is needed."""
+    if world == 1 or dist is None:
+        return local_ms, local_units
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([float(local_units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ------------------------------------------------------------------------------------------------
+def reference_sample(w):
+    """Bounded sample of a workload for the CPU oracle: same kind of problem, fewer units."""
+    from paper_2207_08393_b200 import workloads as wl
+    if w.name == "knee3d":
+        return wl.scaled(w, coils=2, n=(32, w.n[1], w.n[2])), "2 of 8 coils, 32 of 320 readout slabs (32x320x256)"
+    if w.name in ("knee2d", "brain2d"):
+        return wl.scaled(w, batch=1), "batch 1 of %d" % w.batch
+    return w, "whole workload"
+
+
+def make_problem(w, seed_offset=0):
+    from paper_2207_08393_b200 import workloads as wl
+    inp = wl.make_inputs(w, seed_offset)
+    y = wl.standin_kspace(w, inp["mask"], seed_offset)
+    return inp, y
+
+
+def run_reference(args, w):
+    """Times the CPU oracle, as it stands, on a bounded sample (rank 0 only)."""
+    rank, world, _ = dist_setup(args.gpus)
+    if rank != 0:
+        return
+    from oracle import oracle
+    oracle.build()
+    ws, sample_txt = reference_sample(w)
+    inp, y = make_problem(ws)
+    d = oracle.Dims(ws.batch, ws.coils, ws.frames, ws.fft_rank, ws.n, 0, oracle.MASK_READOUT_INVARIANT)
+    cores = oracle.max_threads()
+
+    def step():
+        oracle.dc_forward(inp["x"], y, inp["sens"], inp["mask"], ws.eta, d, nthreads=cores)
+        oracle.dc_vjp(inp["g"], inp["sens"], inp["mask"], ws.eta, d, nthreads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = ws.voxel_coils * args.steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "description": w.description, "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample_txt},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, w):
+    import numpy as np
+    import torch
+    import paper_2207_08393_b200 as g
+
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    g.load_library()
+    peaks = load_peaks()
+
+    inp, y = make_problem(w, seed_offset=rank)
+    tx, tg, ts, tm, ty = (torch.from_numpy(a).to(dev) for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
+    dc = g.DataConsistency(w.batch, w.coils, w.frames, w.fft_rank, w.n)
+    out = torch.empty_like(tx)
+    gin = torch.empty_like(tg)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        dc.forward(tx, ty, ts, tm, w.eta, out)
+        dc.vjp(tg, ts, tm, w.eta, gin)
+
+    flush = None
+    inputs_bytes = sum(t.numel() * t.element_size() for t in (tx, tg, ts, tm, ty))
+    if inputs_bytes < 256 << 20:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # L2 is 126 MB
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- device-resident timed region -------------------------------------------------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = g.gleam_dc_launch_count()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+        local_ms = e0.elapsed_time(e1)
+    else:
+        # small workloads: flush L2 between steps, time each step with its own event pair
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        barrier()
+        for a, b in evs:
+            flush.fill_(1)
+            a.record(stream)
+            step()
+            b.record(stream)
+        barrier()
+        local_ms = sum(a.elapsed_time(b) for a, b in evs)
+    launches = g.gleam_dc_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    total_ms, total_units = aggregate(local_ms, w.voxel_coils * args.steps, world, dist, dev)
+    value = total_units / (total_ms * 1e-3)
+
+    # ---- per-kernel pass (CUDA events around every launch, on the launching stream) ----------
+    prof_steps = min(args.steps, 5)
+    g.gleam_dc_profile_begin()
+    for _ in range(prof_steps):
+        if flush is not None:
+            flush.fill_(1)
+        step()
+    prof = g.gleam_dc_profile_end()
+    kernels = {}
+    for cls, (ms, cnt) in prof.items():
+        per_call = cnt / (2.0 * prof_steps)        # launches per call, averaged over forward and vjp
+        nbytes, flops = kernel_work(cls, w, max(per_call, 1e-9))
+        avg_s = ms * 1e-3 / cnt
+        kernels[cls] = {"launches_per_step": cnt / prof_steps, "ms_per_step": ms / prof_steps, "avg_us": avg_s * 1e6,
+                        "gbs": nbytes / avg_s / 1e9, "tflops": flops / avg_s / 1e12}
+    # forward / vjp split (events around whole calls)
+    ef = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    split = [0.0, 0.0]
+    for _ in range(prof_steps):
+        if flush is not None:
+            flush.fill_(1)
+        ef[0].record(stream); dc.forward(tx, ty, ts, tm, w.eta, out)
+        ef[1].record(stream); dc.vjp(tg, ts, tm, w.eta, gin)
+        ef[2].record(stream); torch.cuda.synchronize()
+        split[0] += ef[0].elapsed_time(ef[1]) / prof_steps
+        split[1] += ef[1].elapsed_time(ef[2]) / prof_steps
+
+    # ---- end to end through the host-buffer entry points --------------------------------------
+    e2e_steps = max(1, min(args.steps, 3 if inputs_bytes > (1 << 30) else 10))
+    hx, hg, hs, hm, hy = (torch.from_numpy(a).pin_memory() for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
+    hout, hgin = torch.empty_like(hx).pin_memory(), torch.empty_like(hg).pin_memory()
+    d_host = g.make_dims(w.batch, w.coils, w.frames, w.fft_rank, w.n, stream=stream)
+    arena = torch.empty(g.gleam_dc_host_arena_size(d_host), dtype=torch.uint8, device=dev)
+
+    def step_host():
+        g.gleam_dc_forward_host(hx, hy, hs, hm, w.eta, hout, d_host, arena)
+        g.gleam_dc_vjp_host(hg, hs, hm, w.eta, hgin, d_host, arena)
+
+    step_host()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        step_host()
+    e1.record(stream)
+    barrier()
+    e2e_ms, e2e_units = aggregate(e0.elapsed_time(e1), w.voxel_coils * e2e_steps, world, dist, dev)
+    nb = lambda t: t.numel() * t.element_size()
+    h2d = nb(hx) + nb(hy) + 2 * nb(hs) + 2 * nb(hm) + nb(hg)
+    d2h = nb(hout) + nb(hgin)
+    # the host path must give the same result as the device path
+    assert torch.equal(hout.to(dev), out) and torch.equal(hgin.to(dev), gin), "host-buffer path differs"
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline --------------------------------------------------------------------------------
+    sm_mhz = peaks["sm_max_mhz"]
+    alu_peak = fp32_peak_tflops(sm_mhz)
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    kd = kernels[dom]
+    t_hbm = kd["gbs"] / peaks["hbm_gbs"]
+    t_alu = kd["tflops"] / alu_peak
+    if t_hbm >= t_alu:
+        roof = {"bound": "hbm", "achieved": kd["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": t_hbm}
+    else:
+        roof = {"bound": "alu", "achieved": kd["tflops"], "peak": alu_peak, "unit": "TFLOP/s", "frac": t_alu}
+    roof.update({"kernel": dom, "peak_source": peaks["source"] + (" copy bandwidth" if roof["bound"] == "hbm" else
+                 " sm_max_mhz x 148 SMs x 128 lanes x 2"), "traffic": TRAFFIC.get((w.name, dom)),
+                 "share_of_step": kd["ms_per_step"] / sum(k["ms_per_step"] for k in kernels.values())})
+    ns = {}
+    for name, with_y, ms in (("forward", True, split[0]), ("vjp", False, split[1])):
+        nbytes, flops = north_star_roofline(w, with_y)
+        t_b, t_f = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (alu_peak * 1e12)
+        ns[name] = {"min_bytes": nbytes, "fft_flops": flops, "hbm_us": t_b * 1e6, "fp32_us": t_f * 1e6,
+                    "measured_us": ms * 1e3, "frac": max(t_b, t_f) / (ms * 1e-3)}
+
+    # ---- CPU baseline: the oracle, once, on the GPU machine's host cores ---------------------------
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import oracle
+        oracle.build()
+        cores = oracle.max_threads()
+        wsamp, sample_txt = (w, "whole workload, 1 step") if w.name != "knee3d" or cores >= 8 else reference_sample(w)
+        if wsamp is not w:
+            inp_c, y_c = make_problem(wsamp)
+        else:
+            inp_c, y_c = inp, y
+        d = oracle.Dims(wsamp.batch, wsamp.coils, wsamp.frames, wsamp.fft_rank, wsamp.n, 0, oracle.MASK_READOUT_INVARIANT)
+        t0 = time.perf_counter()
+        oracle.dc_forward(inp_c["x"], y_c, inp_c["sens"], inp_c["mask"], wsamp.eta, d, nthreads=cores)
+        oracle.dc_vjp(inp_c["g"], inp_c["sens"], inp_c["mask"], wsamp.eta, d, nthreads=cores)
+        dt = time.perf_counter() - t0
+        cpu = {"value": wsamp.voxel_coils / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample_txt,
+               "seconds": dt}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "description": w.description, "step": "1 gleam_dc_forward + 1 gleam_dc_vjp",
+                   "voxel_coils_per_step": w.voxel_coils, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "inputs exceed L2" if flush is None else "256 MB L2 flush before every step"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+        "north_star_roofline": ns,
+        "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
+# an ncu capture, keyed by (workload, kernel class); None until a capture of the current kernel exists.
+TRAFFIC = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="knee3d")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2207_08393_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -117,6 +117,45 @@ GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes);
  */
 GLEAM_API int gleam_dc_length_supported(int32_t n);
 
+/*
+ * Host-buffer variants of the two calls above (no counterpart in the paper: a convenience for
+ * callers whose data lives in host memory).  x, y, sens, mask, out are HOST pointers with the same
+ * layouts; pinned memory makes the copies asynchronous.  `arena` is a DEVICE buffer of at least
+ * gleam_dc_host_arena_size() bytes, 256-byte aligned, that holds the staged inputs, the output and
+ * the workspace; dims->workspace is ignored.  The calls enqueue, on dims->stream, the
+ * host-to-device copies, the kernels and the device-to-host copy of the result, and return
+ * without synchronising: out is valid once the stream has drained.
+ */
+GLEAM_API int gleam_dc_forward_host(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                    void* out, const gleam_dims* dims, void* arena, uint64_t arena_bytes);
+GLEAM_API int gleam_dc_vjp_host(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
+                                const gleam_dims* dims, void* arena, uint64_t arena_bytes);
+GLEAM_API int gleam_dc_host_arena_size(const gleam_dims* dims, uint64_t* bytes);
+
+/*
+ * Measurement aids (no counterpart in the paper).
+ * gleam_dc_launch_count: kernels this library has launched since it was loaded.
+ * gleam_dc_profile_begin / _end: between the two, every kernel launch is bracketed by CUDA events
+ * on its stream; _end waits for the last one and returns, per kernel class GLEAM_K_*, the summed
+ * device time in milliseconds and the number of launches (arrays of n_classes entries).
+ * Profiling creates CUDA events on first use and is meant for benchmarks, not for production.
+ */
+enum {
+    GLEAM_K_PREP_M2 = 0,      /* mask table */
+    GLEAM_K_COL_Z = 1,        /* readout-axis inverse transform of y */
+    GLEAM_K_ROW_FUSED = 2,    /* 2-D one-pass kernel */
+    GLEAM_K_ROW_FWD = 3,      /* sensitivity multiply + transform of the contiguous axis */
+    GLEAM_K_COL_MID_SEP = 4,  /* strided axis forward, mask/residual, inverse (separable path) */
+    GLEAM_K_ROW_INV = 5,      /* inverse of the contiguous axis + coil sum + update */
+    GLEAM_K_COL_MID_FULL = 6, /* same as 4 for a full mask */
+    GLEAM_K_COL_FWD = 7,
+    GLEAM_K_COL_INV = 8,
+    GLEAM_K_CLASSES = 9
+};
+GLEAM_API uint64_t gleam_dc_launch_count(void);
+GLEAM_API int gleam_dc_profile_begin(void);
+GLEAM_API int gleam_dc_profile_end(float* ms, uint32_t* launches, int32_t n_classes);
+
 /* Static, human-readable text for a status code. */
 GLEAM_API const char* gleam_status_string(int status);
 

@@ -28,7 +28,11 @@ GLEAM_MASK_FULL = 0
 GLEAM_MASK_READOUT_INVARIANT = 1
 
 EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam_dc_length_supported",
-           "gleam_status_string", "gleam_version"]
+           "gleam_status_string", "gleam_version", "gleam_dc_forward_host", "gleam_dc_vjp_host",
+           "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end"]
+
+KERNEL_CLASSES = ["prep_m2", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
+                  "col_inv"]
 
 
 class gleam_dims(ctypes.Structure):
@@ -79,6 +83,19 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_status_string.restype = ctypes.c_char_p
         lib.gleam_version.argtypes = []
         lib.gleam_version.restype = i32
+        u64 = ctypes.c_uint64
+        lib.gleam_dc_forward_host.argtypes = [vp, vp, vp, vp, f32, vp, dp, vp, u64]
+        lib.gleam_dc_forward_host.restype = i32
+        lib.gleam_dc_vjp_host.argtypes = [vp, vp, vp, f32, vp, dp, vp, u64]
+        lib.gleam_dc_vjp_host.restype = i32
+        lib.gleam_dc_host_arena_size.argtypes = [dp, ctypes.POINTER(u64)]
+        lib.gleam_dc_host_arena_size.restype = i32
+        lib.gleam_dc_launch_count.argtypes = []
+        lib.gleam_dc_launch_count.restype = u64
+        lib.gleam_dc_profile_begin.argtypes = []
+        lib.gleam_dc_profile_begin.restype = i32
+        lib.gleam_dc_profile_end.argtypes = [ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_uint32), ctypes.c_int32]
+        lib.gleam_dc_profile_end.restype = i32
         _lib = lib
     return _lib
 
@@ -144,6 +161,45 @@ def gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, dims: gleam_dims) -> None:
     """grad_in = grad_out - eta A^H A grad_out  (VJP of Eq. 3 with respect to x)."""
     _check(load_library().gleam_dc_vjp(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
                                         ctypes.byref(dims)))
+
+
+def gleam_dc_host_arena_size(dims: gleam_dims) -> int:
+    out = ctypes.c_uint64(0)
+    _check(load_library().gleam_dc_host_arena_size(ctypes.byref(dims), ctypes.byref(out)))
+    return int(out.value)
+
+
+def gleam_dc_forward_host(x, y, sens, mask, eta, out, dims: gleam_dims, arena, arena_bytes=None) -> None:
+    """Host-buffer variant: x, y, sens, mask, out are host tensors (pinned for asynchronous copies);
+    arena is a device uint8 tensor of gleam_dc_host_arena_size(dims) bytes."""
+    if arena_bytes is None:
+        arena_bytes = arena.numel() * arena.element_size()
+    _check(load_library().gleam_dc_forward_host(_addr(x), _addr(y), _addr(sens), _addr(mask), float(eta), _addr(out),
+                                                 ctypes.byref(dims), _addr(arena), int(arena_bytes)))
+
+
+def gleam_dc_vjp_host(grad_out, sens, mask, eta, grad_in, dims: gleam_dims, arena, arena_bytes=None) -> None:
+    if arena_bytes is None:
+        arena_bytes = arena.numel() * arena.element_size()
+    _check(load_library().gleam_dc_vjp_host(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
+                                             ctypes.byref(dims), _addr(arena), int(arena_bytes)))
+
+
+def gleam_dc_launch_count() -> int:
+    return int(load_library().gleam_dc_launch_count())
+
+
+def gleam_dc_profile_begin() -> None:
+    _check(load_library().gleam_dc_profile_begin())
+
+
+def gleam_dc_profile_end() -> dict:
+    """Returns {kernel class: (milliseconds, launches)} accumulated since gleam_dc_profile_begin()."""
+    n = len(KERNEL_CLASSES)
+    ms = (ctypes.c_float * n)()
+    cnt = (ctypes.c_uint32 * n)()
+    _check(load_library().gleam_dc_profile_end(ms, cnt, n))
+    return {KERNEL_CLASSES[i]: (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
 
 
 class DataConsistency:

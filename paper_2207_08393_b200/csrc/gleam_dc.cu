@@ -13,8 +13,11 @@
 #include "../../include/gleam.h"
 #include "size_ops.cuh"
 
-#include <cstdlib>
+#include <atomic>
 #include <cmath>
+#include <cstdlib>
+#include <mutex>
+#include <vector>
 
 namespace gleam {
 
@@ -124,6 +127,30 @@ static inline float gsign(int n) { return ((n / 2) % 2) ? -1.f : 1.f; }
 
 #define CK(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return GLEAM_ERR_CUDA; } while (0)
 
+// ---- launch counter and optional per-kernel event timing (measurement aid) ----
+static std::atomic<unsigned long long> g_launches{0};
+static std::mutex g_prof_mutex;
+static bool g_prof_on = false;
+static std::vector<cudaEvent_t> g_prof_events;   // event i is recorded just before launch i
+static std::vector<int> g_prof_class;            // kernel class of launch i, -1 = end-of-call marker
+static size_t g_prof_used = 0;
+
+static cudaError_t prof_mark(int cls, cudaStream_t s) {
+    if (cls >= 0) g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!g_prof_on) return cudaSuccess;
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (g_prof_used == g_prof_events.size()) {
+        cudaEvent_t e;
+        cudaError_t r = cudaEventCreate(&e);
+        if (r != cudaSuccess) return r;
+        g_prof_events.push_back(e);
+        g_prof_class.push_back(cls);
+    }
+    g_prof_class[g_prof_used] = cls;
+    return cudaEventRecord(g_prof_events[g_prof_used++], s);
+}
+#define LAUNCH(cls, call) do { CK(prof_mark((cls), s)); CK(call); } while (0)
+
 static int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
                const gleam_dims* d) {
     if (!d) return GLEAM_ERR_NULL_POINTER;
@@ -178,6 +205,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             const long long tot = L.images * pe;
             const int th = 256;
             long long bl = (tot + th - 1) / th; if (bl > 148 * 8) bl = 148 * 8;
+            CK(prof_mark(GLEAM_K_PREP_M2, s));
             prep_m2_kernel<<<(unsigned)bl, th, 0, s>>>(mask, m2, L.images, L.n1, L.n2, L.rank, 1.0f / (float)pe);
             CK(cudaGetLastError());
         }
@@ -189,27 +217,27 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             const int nro = (L.rank == 2) ? L.n1 : L.n0;
             float g = gsign(nro) * gsign(L.n2) * (L.rank == 3 ? gsign(L.n1) : 1.f);
             cz.scale = g / sqrtf((float)nro * (float)pe);
-            CK(((L.rank == 2) ? op1 : op0)->col(COL_Z, cz, s));
+            LAUNCH(GLEAM_K_COL_Z, ((L.rank == 2) ? op1 : op0)->col(COL_Z, cz, s));
         }
         if (L.rank == 2) {
             ra.m2 = m2; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
-            CK(op2->row(ROW_FUSED, ra, s));
+            LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
             cf* W = (cf*)(ws + L.off_W);
             for (int i0 = 0; i0 < L.n0; i0 += L.G) {
                 const int g = (L.n0 - i0 < L.G) ? (L.n0 - i0) : L.G;
                 ra.W = W; ra.rpb = g * L.n1; ra.row0 = i0 * L.n1; ra.nrows = L.images * ra.rpb;
-                CK(op2->row(ROW_FWD, ra, s));
+                LAUNCH(GLEAM_K_ROW_FWD, op2->row(ROW_FWD, ra, s));
                 ColArgs cm = ca;
                 cm.W = W; cm.m2 = m2; cm.zin = z; cm.es = L.n2; cm.nouter = L.units * g; cm.G = g; cm.i0_start = i0;
-                CK(op1->col(COL_MID_SEP, cm, s));
-                CK(op2->row(ROW_INV, ra, s));
+                LAUNCH(GLEAM_K_COL_MID_SEP, op1->col(COL_MID_SEP, cm, s));
+                LAUNCH(GLEAM_K_ROW_INV, op2->row(ROW_INV, ra, s));
             }
         }
     } else {
         cf* W = (cf*)(ws + L.off_W);
         ra.W = W; ra.rpb = L.n0 * L.n1; ra.row0 = 0; ra.nrows = L.images * ra.rpb;
-        CK(op2->row(ROW_FWD, ra, s));
+        LAUNCH(GLEAM_K_ROW_FWD, op2->row(ROW_FWD, ra, s));
         float g = gsign(L.n2) * gsign(L.n1) * (L.rank == 3 ? gsign(L.n0) : 1.f);
         const double ntot = (L.rank == 3) ? (double)L.V : (double)L.n1 * L.n2;
         ColArgs cm = ca;
@@ -217,17 +245,18 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
         cm.scale = g / (float)sqrt(ntot); cm.scale2 = (float)(1.0 / ntot);
         if (L.rank == 2) {
             cm.es = L.n2; cm.nouter = L.units;
-            CK(op1->col(COL_MID_FULL, cm, s));
+            LAUNCH(GLEAM_K_COL_MID_FULL, op1->col(COL_MID_FULL, cm, s));
         } else {
             ColArgs c1 = ca;
             c1.W = W; c1.es = L.n2; c1.nouter = L.units * L.n0;
-            CK(op1->col(COL_FWD, c1, s));
+            LAUNCH(GLEAM_K_COL_FWD, op1->col(COL_FWD, c1, s));
             cm.es = L.n1 * L.n2; cm.nouter = L.units;
-            CK(op0->col(COL_MID_FULL, cm, s));
-            CK(op1->col(COL_INV, c1, s));
+            LAUNCH(GLEAM_K_COL_MID_FULL, op0->col(COL_MID_FULL, cm, s));
+            LAUNCH(GLEAM_K_COL_INV, op1->col(COL_INV, c1, s));
         }
-        CK(op2->row(ROW_INV, ra, s));
+        LAUNCH(GLEAM_K_ROW_INV, op2->row(ROW_INV, ra, s));
     }
+    CK(prof_mark(-1, s));
     return GLEAM_OK;
 }
 
@@ -276,5 +305,95 @@ GLEAM_API const char* gleam_status_string(int status) {
 }
 
 GLEAM_API int gleam_version(void) { return GLEAM_VERSION; }
+
+GLEAM_API uint64_t gleam_dc_launch_count(void) { return gleam::g_launches.load(); }
+
+GLEAM_API int gleam_dc_profile_begin(void) {
+    std::lock_guard<std::mutex> lock(gleam::g_prof_mutex);
+    gleam::g_prof_on = true;
+    gleam::g_prof_used = 0;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_profile_end(float* ms, uint32_t* launches, int32_t n_classes) {
+    using namespace gleam;
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    g_prof_on = false;
+    if (!ms || !launches) return GLEAM_ERR_NULL_POINTER;
+    for (int i = 0; i < n_classes; ++i) { ms[i] = 0.f; launches[i] = 0; }
+    if (g_prof_used == 0) return GLEAM_OK;
+    if (cudaEventSynchronize(g_prof_events[g_prof_used - 1]) != cudaSuccess) return GLEAM_ERR_CUDA;
+    for (size_t i = 0; i + 1 < g_prof_used; ++i) {
+        const int cls = g_prof_class[i];
+        if (cls < 0 || cls >= n_classes) continue;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, g_prof_events[i], g_prof_events[i + 1]) != cudaSuccess) return GLEAM_ERR_CUDA;
+        ms[cls] += t;
+        launches[cls] += 1;
+    }
+    g_prof_used = 0;
+    return GLEAM_OK;
+}
+
+static int host_arena_layout(const gleam_dims* d, uint64_t off[7], uint64_t sz[6]) {
+    gleam::Layout L;
+    int rc = gleam::make_layout(d, true, &L);
+    if (rc != GLEAM_OK) return rc;
+    const long long pe = (L.rank == 2) ? L.n2 : (long long)L.n1 * L.n2;
+    sz[0] = (uint64_t)L.images * L.V * 8;                                   // x / grad_out
+    sz[1] = (uint64_t)L.units * L.V * 8;                                    // y
+    sz[2] = (uint64_t)L.B * L.C * L.Ts * L.V * 8;                           // sens
+    sz[3] = (uint64_t)L.images * (L.separable ? pe : L.V) * 4;              // mask
+    sz[4] = sz[0];                                                          // out
+    sz[5] = L.total;                                                        // workspace
+    uint64_t o = 0;
+    for (int i = 0; i < 6; ++i) { off[i] = o; o = gleam::align_up(o + sz[i], 256); }
+    off[6] = o;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_host_arena_size(const gleam_dims* dims, uint64_t* bytes) {
+    if (!dims || !bytes) return GLEAM_ERR_NULL_POINTER;
+    uint64_t off[7], sz[6];
+    int rc = host_arena_layout(dims, off, sz);
+    if (rc != GLEAM_OK) return rc;
+    *bytes = off[6];
+    return GLEAM_OK;
+}
+
+static int run_host(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
+                    const gleam_dims* dims, void* arena, uint64_t arena_bytes) {
+    if (!dims || !x || !sens || !mask || !out || !arena) return GLEAM_ERR_NULL_POINTER;
+    if (((uintptr_t)arena & 255) != 0) return GLEAM_ERR_BAD_DIMS;
+    uint64_t off[7], sz[6];
+    int rc = host_arena_layout(dims, off, sz);
+    if (rc != GLEAM_OK) return rc;
+    if (arena_bytes < off[6]) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    char* a = (char*)arena;
+    cudaStream_t s = (cudaStream_t)dims->stream;
+    const void* src[4] = {x, y, sens, mask};
+    for (int i = 0; i < 4; ++i) {
+        if (!src[i]) continue;
+        if (cudaMemcpyAsync(a + off[i], src[i], sz[i], cudaMemcpyHostToDevice, s) != cudaSuccess) return GLEAM_ERR_CUDA;
+    }
+    gleam_dims d = *dims;
+    d.workspace = a + off[5];
+    d.workspace_bytes = sz[5];
+    rc = gleam::run(a + off[0], y ? a + off[1] : nullptr, a + off[2], (const float*)(a + off[3]), eta, a + off[4], &d);
+    if (rc != GLEAM_OK) return rc;
+    if (cudaMemcpyAsync(out, a + off[4], sz[4], cudaMemcpyDeviceToHost, s) != cudaSuccess) return GLEAM_ERR_CUDA;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_forward_host(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                    void* out, const gleam_dims* dims, void* arena, uint64_t arena_bytes) {
+    if (!y) return GLEAM_ERR_NULL_POINTER;
+    return run_host(x, y, sens, mask, eta, out, dims, arena, arena_bytes);
+}
+
+GLEAM_API int gleam_dc_vjp_host(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
+                                const gleam_dims* dims, void* arena, uint64_t arena_bytes) {
+    return run_host(grad_out, nullptr, sens, mask, eta, grad_in, dims, arena, arena_bytes);
+}
 
 }  // extern "C"

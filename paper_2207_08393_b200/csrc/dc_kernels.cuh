@@ -23,7 +23,7 @@ struct RowArgs {
     const cf* x;        // image-domain input (B,T,n0,n1,n2)
     const cf* sens;     // (B,C,[T],n0,n1,n2)
     cf* out;            // (B,T,n0,n1,n2)
-    const float* m2;    // ROW_FUSED: (B,T,n2) shifted mask^2 / n2
+    const float* mask;  // ROW_FUSED: readout-invariant mask (B,T,n2)
     const cf* z;        // ROW_FUSED: (B,C,T,n1,n2) shifted, signed, masked R^H y; may be null
     cf* W;              // workspace (unit, rpb, n2)
     float eta;
@@ -39,15 +39,14 @@ struct ColArgs {
     const cf* y;        // COL_Z input / COL_MID_FULL measurements (B,C,T,V)
     cf* z;              // COL_Z output
     const cf* zin;      // COL_MID_SEP: z table (unit, n0, n1, n2)
-    const float* mask;  // COL_Z: readout-invariant mask; COL_MID_FULL: full mask (B,T,V)
-    const float* m2;    // COL_MID_SEP: (B,T,n1,n2) shifted mask^2 / (n1 n2)
+    const float* mask;  // COL_Z, COL_MID_SEP: readout-invariant mask; COL_MID_FULL: full mask (B,T,V)
     int es;             // element stride of the transformed axis = lines per outer index
     long long nouter;   // outer indices
     int C, T;
     int rank, n0, n1, n2;
     int G, i0_start;    // COL_MID_SEP chunk: slabs in the chunk, first slab
     float scale;        // COL_Z: g_ro g_pe / sqrt(N_ro N_pe);  COL_MID_FULL: g / sqrt(Ntot)
-    float scale2;       // COL_MID_FULL: 1 / Ntot
+    float scale2;       // COL_MID_FULL: 1 / Ntot;  COL_MID_SEP: 1 / (n1 n2)
 };
 
 __device__ __forceinline__ int shift_half(int k, int n) { int h = n >> 1; return k >= n - h ? k - (n - h) : k + h; }
@@ -84,40 +83,72 @@ row_kernel(const RowArgs a) {
 #pragma unroll
         for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
     }
-    if (act0) {
+    if (MODE != ROW_INV) {
+        if (act0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) xv[m] = a.x[x_off + d.j0 + P::BF0 * m];
+            for (int m = 0; m < R0; ++m) xv[m] = a.x[x_off + d.j0 + P::BF0 * m];
+        }
     }
     float m2v[RL];
     if (MODE == ROW_FUSED) {
         if (actL) {
 #pragma unroll
-            for (int k = 0; k < RL; ++k) m2v[k] = a.m2[btL * N + d.jL + P::BFL * k];
+            for (int k = 0; k < RL; ++k) {
+                const float mv = a.mask[btL * N + shift_half(d.jL + P::BFL * k, N)];
+                m2v[k] = mv * mv * (1.0f / N);
+            }
         }
     }
 
+    // per-coil strides (elements); the loads of coil c+1 are issued before the arithmetic of coil c
+    const long long s_stride = (long long)a.Ts * a.RPB * N;
+    const long long s_base = (((long long)(b0 * a.C) * a.Ts + (a.Ts > 1 ? t0 : 0)) * a.RPB + a.row0 + ri0) * N + d.j0;
+    const long long k_stride = (long long)a.T * ((MODE == ROW_FUSED) ? a.RPB : a.rpb) * N;
+    const long long k_base = (MODE == ROW_FUSED)
+        ? (((long long)(bL * a.C) * a.T + tL) * a.RPB + a.row0 + riL) * N + d.jL
+        : (((long long)(bL * a.C) * a.T + tL) * a.rpb + riL) * N + d.jL;
+    const bool use_z = (MODE == ROW_FUSED) && (a.z != nullptr);
+
+    cf s_cur[R0], s_nxt[R0];      // sensitivities of this / the next coil (n-distribution)
+    cf k_cur[RL], k_nxt[RL];      // z table (ROW_FUSED) or workspace (ROW_INV) values (k-distribution)
+    auto load_s = [&](cf (&dst)[R0], int c) {
+        if (act0) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) dst[m] = a.sens[s_base + c * s_stride + P::BF0 * m];
+        }
+    };
+    auto load_k = [&](cf (&dst)[RL], int c) {
+        if (actL) {
+            const cf* src = (MODE == ROW_FUSED) ? a.z : a.W;
+#pragma unroll
+            for (int k = 0; k < RL; ++k) dst[k] = src[k_base + c * k_stride + P::BFL * k];
+        }
+    };
+    load_s(s_cur, 0);
+    if (MODE == ROW_INV || use_z) load_k(k_cur, 0);
+
     for (int c = 0; c < a.C; ++c) {
-        const long long s_off = (((long long)(b0 * a.C + c) * a.Ts + (a.Ts > 1 ? t0 : 0)) * a.RPB + a.row0 + ri0) * N;
+        if (c + 1 < a.C) {
+            load_s(s_nxt, c + 1);
+            if (MODE == ROW_INV || use_z) load_k(k_nxt, c + 1);
+        }
         cf v[R0], u[RL];
         if (MODE != ROW_INV) {
             if (act0) {
 #pragma unroll
-                for (int m = 0; m < R0; ++m) v[m] = cmul(a.sens[s_off + d.j0 + P::BF0 * m], xv[m]);
+                for (int m = 0; m < R0; ++m) v[m] = cmul(s_cur[m], xv[m]);
             } else {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) v[m] = make_float2(0.f, 0.f);
             }
-            E::forward(v, u, tw, d, smem);
+            E::forward(v, u, tw, d, smem, (MODE == ROW_FWD) ? (c & 1) : 0);
         }
         if (MODE == ROW_FUSED) {
             if (actL) {
-                if (a.z) {
-                    const long long z_off = (((long long)(bL * a.C + c) * a.T + tL) * a.RPB + a.row0 + riL) * N;
+                if (use_z) {
 #pragma unroll
-                    for (int k = 0; k < RL; ++k) {
-                        const cf zz = a.z[z_off + d.jL + P::BFL * k];
-                        u[k] = make_float2(fmaf(m2v[k], u[k].x, -zz.x), fmaf(m2v[k], u[k].y, -zz.y));
-                    }
+                    for (int k = 0; k < RL; ++k)
+                        u[k] = make_float2(fmaf(m2v[k], u[k].x, -k_cur[k].x), fmaf(m2v[k], u[k].y, -k_cur[k].y));
                 } else {
 #pragma unroll
                     for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], m2v[k]);
@@ -125,32 +156,36 @@ row_kernel(const RowArgs a) {
             }
         } else if (MODE == ROW_FWD) {
             if (actL) {
-                const long long w_off = (((long long)(bL * a.C + c) * a.T + tL) * a.rpb + riL) * N;
 #pragma unroll
-                for (int k = 0; k < RL; ++k) a.W[w_off + d.jL + P::BFL * k] = u[k];
+                for (int k = 0; k < RL; ++k) a.W[k_base + c * k_stride + P::BFL * k] = u[k];
             }
         } else {  // ROW_INV
-            if (actL) {
-                const long long w_off = (((long long)(bL * a.C + c) * a.T + tL) * a.rpb + riL) * N;
 #pragma unroll
-                for (int k = 0; k < RL; ++k) u[k] = a.W[w_off + d.jL + P::BFL * k];
-            }
+            for (int k = 0; k < RL; ++k) u[k] = k_cur[k];
         }
         if (MODE != ROW_FWD) {
-            E::inverse(u, v, tw, d, smem);
+            E::inverse(u, v, tw, d, smem, (MODE == ROW_INV) ? (c & 1) : 0);
             if (act0) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
-                    const cf s = a.sens[s_off + d.j0 + P::BF0 * m];
+                    const cf sv = s_cur[m];
                     // acc += conj(s) * v
-                    acc[m].x = fmaf(s.x, v[m].x, fmaf(s.y, v[m].y, acc[m].x));
-                    acc[m].y = fmaf(s.x, v[m].y, fmaf(-s.y, v[m].x, acc[m].y));
+                    acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
+                    acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
                 }
             }
         }
+#pragma unroll
+        for (int m = 0; m < R0; ++m) s_cur[m] = s_nxt[m];
+#pragma unroll
+        for (int k = 0; k < RL; ++k) k_cur[k] = k_nxt[k];
     }
     if (MODE != ROW_FWD) {
         if (act0) {
+            if (MODE == ROW_INV) {
+#pragma unroll
+                for (int m = 0; m < R0; ++m) xv[m] = a.x[x_off + d.j0 + P::BF0 * m];
+            }
 #pragma unroll
             for (int m = 0; m < R0; ++m)
                 a.out[x_off + d.j0 + P::BF0 * m] =
@@ -252,12 +287,13 @@ col_kernel(const ColArgs a) {
             const int t = (int)(unit % a.T);
             const int b = (int)(unit / ((long long)a.C * a.T));
             const long long pe = (long long)a.n1 * a.n2;
-            const float* m2 = a.m2 + ((long long)b * a.T + t) * pe + i;
+            const float* mk = a.mask + ((long long)b * a.T + t) * pe + shift_half(i, a.n2);
             const cf* zz = a.zin ? a.zin + (unit * a.n0 + a.i0_start + gi) * pe + i : nullptr;
 #pragma unroll
             for (int k = 0; k < RL; ++k) {
                 const long long kk = (long long)(d.jL + P::BFL * k) * a.n2;
-                const float w = m2[kk];
+                const float mv = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
+                const float w = mv * mv * a.scale2;
                 if (zz) {
                     const cf q = zz[kk];
                     u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));

@@ -35,21 +35,17 @@ struct Plan {
     static constexpr int LSZ = 2 * BUF;            // two buffers per line
 };
 
-// exp(-2 pi i e / n) for 0 <= e < n, accurate to float rounding (octant reduction in integers)
-__device__ __forceinline__ cf unit_root_fwd(int e, int n) {
-    // angle fraction e/n of a turn
-    bool neg_sin = false, neg_cos = false, swap = false;
-    long long p = e, q = n;
-    if (2 * p > q) { p = q - p; neg_sin = true; }          // a -> 2pi - a
-    if (4 * p > q) { p = q - 2 * p; q = 2 * q; neg_cos = true; }   // a -> pi - a   (a = 2 pi p / q)
-    if (8 * p > q) { p = q - 4 * p; q = 4 * q; swap = true; }      // a -> pi/2 - a
-    float s, c;
-    sincospif(2.0f * (float)p / (float)q, &s, &c);
-    if (swap) { float t = s; s = c; c = t; }
-    if (neg_cos) c = -c;
-    if (neg_sin) s = -s;
-    return make_float2(c, -s);     // forward sign: exp(-i a)
+// exp(-2 pi i e / N), e = 0..N-1, evaluated at compile time in double precision and stored as a
+// device-resident constant table (a few KB per length, read through L1).
+template <int N> struct RootTable { cf v[N]; };
+template <int N> constexpr RootTable<N> make_root_table() {
+    RootTable<N> t{};
+    for (int e = 0; e < N; ++e) t.v[e] = cf{float(ct::cos2pi(e, N)), float(-ct::sin2pi(e, N))};
+    return t;
 }
+template <int N> __device__ const RootTable<N> g_roots = make_root_table<N>();
+
+template <int N> __device__ __forceinline__ cf unit_root_fwd(int e) { return g_roots<N>.v[e]; }
 
 template <class P, bool COL, int L>
 struct LineFFT {
@@ -87,24 +83,28 @@ struct LineFFT {
     __device__ __forceinline__ static void make_tw(const Ids& d, Tw& tw) {
         if (S >= 2) {
 #pragma unroll
-            for (int k = 0; k < R0; ++k) tw.t0[k] = unit_root_fwd((d.j0 * k) % N, N);
+            for (int k = 0; k < R0; ++k) tw.t0[k] = unit_root_fwd<N>((d.j0 * k) % N);
         }
         if (S == 3) {
             const int t = d.j1 % P::N2;
 #pragma unroll
-            for (int k = 0; k < R1; ++k) tw.t1[k] = unit_root_fwd((t * k) % P::N1, P::N1);
+            for (int k = 0; k < R1; ++k) tw.t1[k] = unit_root_fwd<(P::S == 3 ? P::N1 : 1)>(P::S == 3 ? (t * k) % P::N1 : 0);
         }
     }
 
     // v: n-distribution of the first-stage thread; u: k-distribution of the last-stage thread
-    __device__ __forceinline__ static void forward(cf (&v)[R0], cf (&u)[RL], const Tw& tw, const Ids& d, cf* sm) {
+    // flip = 1 swaps the two exchange buffers of a two-stage plan.  A loop that calls only forward()
+    // (or only inverse()) must alternate flip from one call to the next: with a single barrier per
+    // call, the buffer written now must not be the one other threads may still be reading.
+    __device__ __forceinline__ static void forward(cf (&v)[R0], cf (&u)[RL], const Tw& tw, const Ids& d, cf* sm,
+                                                   int flip = 0) {
         if (S == 1) {
             Dft<R0, -1>::run(v);
 #pragma unroll
             for (int k = 0; k < RL; ++k) u[k] = v[k % R0];
             return;
         }
-        cf* X = sm;
+        cf* X = sm + ((S == 2 && flip) ? (COL ? L * P::BUF : P::BUF) : 0);
         cf* Y = sm + (COL ? L * P::BUF : P::BUF);
         if (d.a0) {
             Dft<R0, -1>::run(v);
@@ -146,7 +146,8 @@ struct LineFFT {
     // mirror image of forward(): u (k-distribution) -> v (n-distribution), unscaled inverse.
     // Buffer use: two-stage plans exchange through Y (X may still be read by forward());
     // three-stage plans go through X then Y.
-    __device__ __forceinline__ static void inverse(cf (&u)[RL], cf (&v)[R0], const Tw& tw, const Ids& d, cf* sm) {
+    __device__ __forceinline__ static void inverse(cf (&u)[RL], cf (&v)[R0], const Tw& tw, const Ids& d, cf* sm,
+                                                   int flip = 0) {
         if (S == 1) {
 #pragma unroll
             for (int k = 0; k < R0; ++k) v[k] = u[k % RL];
@@ -154,7 +155,7 @@ struct LineFFT {
             return;
         }
         cf* X = sm;
-        cf* Y = sm + (COL ? L * P::BUF : P::BUF);
+        cf* Y = sm + ((S == 2 && flip) ? 0 : (COL ? L * P::BUF : P::BUF));
         if (S == 3) {
             if (d.aL) {
                 Dft<RL, +1>::run(u);

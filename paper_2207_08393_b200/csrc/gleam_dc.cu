@@ -21,33 +21,16 @@
 
 namespace gleam {
 
-#define GLEAM_SIZE(N, R0, R1, R2, LR, LC) extern const SizeOps size_ops_##N;
+#define GLEAM_SIZE(N, A0, A1, A2, LR, B0, B1, B2, LC) extern const SizeOps size_ops_##N;
 #include "sizes.def"
 #undef GLEAM_SIZE
 
 static const SizeOps* find_size(int n) {
     switch (n) {
-#define GLEAM_SIZE(N, R0, R1, R2, LR, LC) case N: return &size_ops_##N;
+#define GLEAM_SIZE(N, A0, A1, A2, LR, B0, B1, B2, LC) case N: return &size_ops_##N;
 #include "sizes.def"
 #undef GLEAM_SIZE
         default: return nullptr;
-    }
-}
-
-// shifted mask^2 * scale table for the separable paths:  m2[bt][k] = M[bt][sh(k)]^2 * scale
-__global__ void prep_m2_kernel(const float* __restrict__ mask, float* __restrict__ m2, long long nbt,
-                               int n1, int n2, int rank, float scale) {
-    const long long pe = (rank == 2) ? n2 : (long long)n1 * n2;
-    const long long tot = nbt * pe;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < tot;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const long long bt = idx / pe;
-        const int p = (int)(idx % pe);
-        int src;
-        if (rank == 2) src = shift_half(p, n2);
-        else src = shift_half(p / n2, n1) * n2 + shift_half(p % n2, n2);
-        const float mv = mask[bt * pe + src];
-        m2[idx] = mv * mv * scale;
     }
 }
 
@@ -59,7 +42,7 @@ struct Layout {
     long long V, units, images;
     bool separable;
     // workspace (byte offsets)
-    uint64_t off_m2, off_z, off_W, total;
+    uint64_t off_z, off_W, total;
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
@@ -83,10 +66,9 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     if (L->V > (1ll << 40) || L->units * L->V > (1ll << 46)) return GLEAM_ERR_BAD_DIMS;
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
-    L->off_m2 = L->off_z = L->off_W = 0; L->G = 0;
+    L->off_z = L->off_W = 0; L->G = 0;
     if (L->separable) {
         const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
-        L->off_m2 = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(float), 256);
         if (with_y) { L->off_z = off; off = align_up(off + (uint64_t)L->units * L->V * sizeof(cf), 256); }
         if (L->rank == 3) {
             const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
@@ -199,16 +181,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
     ca.C = L.C; ca.T = L.T; ca.rank = L.rank; ca.n0 = L.n0; ca.n1 = L.n1; ca.n2 = L.n2;
 
     if (L.separable) {
-        float* m2 = (float*)(ws + L.off_m2);
         cf* z = y ? (cf*)(ws + L.off_z) : nullptr;
-        {
-            const long long tot = L.images * pe;
-            const int th = 256;
-            long long bl = (tot + th - 1) / th; if (bl > 148 * 8) bl = 148 * 8;
-            CK(prof_mark(GLEAM_K_PREP_M2, s));
-            prep_m2_kernel<<<(unsigned)bl, th, 0, s>>>(mask, m2, L.images, L.n1, L.n2, L.rank, 1.0f / (float)pe);
-            CK(cudaGetLastError());
-        }
         if (y) {
             // z table: inverse transform of y along the readout axis, at sampled positions
             ColArgs cz = ca;
@@ -220,7 +193,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             LAUNCH(GLEAM_K_COL_Z, ((L.rank == 2) ? op1 : op0)->col(COL_Z, cz, s));
         }
         if (L.rank == 2) {
-            ra.m2 = m2; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
+            ra.mask = mask; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
             cf* W = (cf*)(ws + L.off_W);
@@ -229,7 +202,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
                 ra.W = W; ra.rpb = g * L.n1; ra.row0 = i0 * L.n1; ra.nrows = L.images * ra.rpb;
                 LAUNCH(GLEAM_K_ROW_FWD, op2->row(ROW_FWD, ra, s));
                 ColArgs cm = ca;
-                cm.W = W; cm.m2 = m2; cm.zin = z; cm.es = L.n2; cm.nouter = L.units * g; cm.G = g; cm.i0_start = i0;
+                cm.W = W; cm.mask = mask; cm.scale2 = 1.0f / (float)pe; cm.zin = z; cm.es = L.n2; cm.nouter = L.units * g; cm.G = g; cm.i0_start = i0;
                 LAUNCH(GLEAM_K_COL_MID_SEP, op1->col(COL_MID_SEP, cm, s));
                 LAUNCH(GLEAM_K_ROW_INV, op2->row(ROW_INV, ra, s));
             }

@@ -2,9 +2,9 @@
 #include "size_ops.cuh"
 
 namespace gleam {
-#define GLEAM_SIZE(N, R0, R1, R2, LR, LC) \
-    extern const SizeOps size_ops_##N = {N, &SizeImpl<Plan<N, R0, R1, R2>, LR, LC>::row, \
-                                         &SizeImpl<Plan<N, R0, R1, R2>, LR, LC>::col};
+#define GLEAM_SIZE(N, A0, A1, A2, LR, B0, B1, B2, LC) \
+    extern const SizeOps size_ops_##N = {N, &SizeImpl<Plan<N, A0, A1, A2>, LR, Plan<N, B0, B1, B2>, LC>::row, \
+                                         &SizeImpl<Plan<N, A0, A1, A2>, LR, Plan<N, B0, B1, B2>, LC>::col};
 #include "sizes.def"
 #undef GLEAM_SIZE
 }  // namespace gleam

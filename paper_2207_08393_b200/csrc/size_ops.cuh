@@ -48,7 +48,7 @@ inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
     return cudaGetLastError();
 }
 
-template <class P, int LR, int LC>
+template <class P, int LR, class PC, int LC>
 struct SizeImpl {
     static cudaError_t row(int mode, const RowArgs& a, cudaStream_t s) {
         switch (mode) {
@@ -60,11 +60,11 @@ struct SizeImpl {
     }
     static cudaError_t col(int mode, const ColArgs& a, cudaStream_t s) {
         switch (mode) {
-            case COL_Z:        return launch_col<P, LC, COL_Z>(a, s);
-            case COL_MID_SEP:  return launch_col<P, LC, COL_MID_SEP>(a, s);
-            case COL_MID_FULL: return launch_col<P, LC, COL_MID_FULL>(a, s);
-            case COL_FWD:      return launch_col<P, LC, COL_FWD>(a, s);
-            case COL_INV:      return launch_col<P, LC, COL_INV>(a, s);
+            case COL_Z:        return launch_col<PC, LC, COL_Z>(a, s);
+            case COL_MID_SEP:  return launch_col<PC, LC, COL_MID_SEP>(a, s);
+            case COL_MID_FULL: return launch_col<PC, LC, COL_MID_FULL>(a, s);
+            case COL_FWD:      return launch_col<PC, LC, COL_FWD>(a, s);
+            case COL_INV:      return launch_col<PC, LC, COL_INV>(a, s);
         }
         return cudaErrorInvalidValue;
     }

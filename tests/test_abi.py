@@ -57,7 +57,7 @@ def test_workspace_size_formula(lib):
     # readout-invariant 2-D: mask table + z table
     d = g.make_dims(4, 15, 1, 2, (1, 640, 368))
     ws = g.gleam_dc_workspace_size(d)
-    assert ws >= 4 * 368 * 4 + 4 * 15 * 640 * 368 * 8
+    assert ws >= 4 * 15 * 640 * 368 * 8
     # full mask: one coil-volume workspace
     d = g.make_dims(1, 8, 1, 3, (320, 320, 256), mask_kind=g.GLEAM_MASK_FULL)
     assert g.gleam_dc_workspace_size(d) >= 8 * 320 * 320 * 256 * 8
@@ -93,11 +93,11 @@ def test_null_pointers_and_small_workspace(lib):
         g.gleam_dc_forward(8, None, 8, 8, 1.0, 8, d)            # forward needs y
     assert e.value.status == binding.GLEAM_ERR_NULL_POINTER
     with pytest.raises(g.GleamError) as e:
-        g.gleam_dc_vjp(1 << 20, 2 << 20, 3 << 20, 1.0, 4 << 20, d)   # no workspace given
+        g.gleam_dc_forward(1 << 20, 2 << 20, 3 << 20, 4 << 20, 1.0, 5 << 20, d)   # no workspace given
     assert e.value.status == binding.GLEAM_ERR_NULL_POINTER
     d = g.make_dims(1, 2, 1, 2, (1, 64, 64), workspace=1 << 30, workspace_bytes=16)
     with pytest.raises(g.GleamError) as e:
-        g.gleam_dc_vjp(1 << 20, 2 << 20, 3 << 20, 1.0, 4 << 20, d)
+        g.gleam_dc_forward(1 << 20, 2 << 20, 3 << 20, 4 << 20, 1.0, 5 << 20, d)
     assert e.value.status == binding.GLEAM_ERR_WORKSPACE_TOO_SMALL
 
 

@@ -133,6 +133,31 @@ GLEAM_API int gleam_dc_vjp_host(const void* grad_out, const void* sens, const fl
 GLEAM_API int gleam_dc_host_arena_size(const gleam_dims* dims, uint64_t* bytes);
 
 /*
+ * gleam_dc_forward_static: gleam_dc_forward for callers that must not allocate device memory.
+ * (The paper has no counterpart; this is a deployment convenience.)  Some users of this library
+ * run where cudaMalloc is off the table: a reconstruction service whose device memory was handed
+ * out in full to a framework's caching allocator at start-up, a plug-in that may touch only the
+ * buffers its host application passes in, a real-time loop in which an allocation's implicit
+ * device synchronisation is unacceptable.  For them the scratch that gleam_dc_forward takes from
+ * dims->workspace lives inside the library instead, in one fixed device array of
+ * gleam_dc_static_scratch_bytes() bytes (64 MiB) that every GPU loading the library keeps until
+ * the process exits.  dims->workspace and dims->workspace_bytes are ignored; inputs and the
+ * output are still the caller's device buffers, with the layouts and rules of gleam_dc_forward.
+ *   - Problems whose scratch need (gleam_dc_workspace_size) exceeds the array return
+ *     GLEAM_ERR_WORKSPACE_TOO_SMALL and launch nothing.
+ *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls share the one array, which keeps whatever the previous call left in it; the
+ *     kernels write every scratch element before reading it, so no clearing is needed.  Two calls
+ *     whose GPU work overlaps (different streams, or different host threads on one device) race on
+ *     the array and give undefined results: order them on one stream or with events.
+ */
+GLEAM_API int gleam_dc_forward_static(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                      void* out, const gleam_dims* dims);
+GLEAM_API uint64_t gleam_dc_static_scratch_bytes(void);
+
+/*
  * Measurement aids (no counterpart in the paper).
  * gleam_dc_launch_count: kernels this library has launched since it was loaded.
  * gleam_dc_profile_begin / _end: between the two, every kernel launch is bracketed by CUDA events

@@ -29,7 +29,8 @@ GLEAM_MASK_READOUT_INVARIANT = 1
 
 EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam_dc_length_supported",
            "gleam_status_string", "gleam_version", "gleam_dc_forward_host", "gleam_dc_vjp_host",
-           "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end"]
+           "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end",
+           "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes"]
 
 KERNEL_CLASSES = ["prep_m2", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
                   "col_inv"]
@@ -90,6 +91,10 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_dc_vjp_host.restype = i32
         lib.gleam_dc_host_arena_size.argtypes = [dp, ctypes.POINTER(u64)]
         lib.gleam_dc_host_arena_size.restype = i32
+        lib.gleam_dc_forward_static.argtypes = [vp, vp, vp, vp, f32, vp, dp]
+        lib.gleam_dc_forward_static.restype = i32
+        lib.gleam_dc_static_scratch_bytes.argtypes = []
+        lib.gleam_dc_static_scratch_bytes.restype = u64
         lib.gleam_dc_launch_count.argtypes = []
         lib.gleam_dc_launch_count.restype = u64
         lib.gleam_dc_profile_begin.argtypes = []
@@ -183,6 +188,17 @@ def gleam_dc_vjp_host(grad_out, sens, mask, eta, grad_in, dims: gleam_dims, aren
         arena_bytes = arena.numel() * arena.element_size()
     _check(load_library().gleam_dc_vjp_host(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
                                              ctypes.byref(dims), _addr(arena), int(arena_bytes)))
+
+
+def gleam_dc_static_scratch_bytes() -> int:
+    return int(load_library().gleam_dc_static_scratch_bytes())
+
+
+def gleam_dc_forward_static(x, y, sens, mask, eta, out, dims: gleam_dims) -> None:
+    """gleam_dc_forward with the library's own fixed scratch array instead of dims.workspace, for
+    callers that cannot allocate device memory.  Calls whose GPU work overlaps race on that array."""
+    _check(load_library().gleam_dc_forward_static(_addr(x), _addr(y), _addr(sens), _addr(mask), float(eta),
+                                                   _addr(out), ctypes.byref(dims)))
 
 
 def gleam_dc_launch_count() -> int:

@@ -279,6 +279,49 @@ GLEAM_API const char* gleam_status_string(int status) {
 
 GLEAM_API int gleam_version(void) { return GLEAM_VERSION; }
 
+// ---- fixed scratch for callers that cannot allocate device memory ----
+// One array per GPU that loads this library, resident until the process exits.
+#define GLEAM_STATIC_SCRATCH_BYTES (64ull << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[GLEAM_STATIC_SCRATCH_BYTES];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address the GPU can
+// use, so the device address is looked up once per device (with that device current) and cached.
+static int static_scratch_address(void** out) {
+    enum { MAX_DEVICES = 64 };
+    static void* cache[MAX_DEVICES] = {nullptr};
+    static std::mutex mtx;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return GLEAM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mtx);
+    if (!cache[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return GLEAM_ERR_CUDA; }
+        cache[dev] = p;
+    }
+    *out = cache[dev];
+    return GLEAM_OK;
+}
+
+GLEAM_API uint64_t gleam_dc_static_scratch_bytes(void) { return GLEAM_STATIC_SCRATCH_BYTES; }
+
+GLEAM_API int gleam_dc_forward_static(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                      void* out, const gleam_dims* dims) {
+    if (!dims || !y) return GLEAM_ERR_NULL_POINTER;
+    gleam::Layout L;
+    int rc = gleam::make_layout(dims, true, &L);
+    if (rc != GLEAM_OK) return rc;
+    if (L.total > GLEAM_STATIC_SCRATCH_BYTES) return GLEAM_ERR_WORKSPACE_TOO_SMALL;   // problem too large for the fixed scratch
+    void* scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != GLEAM_OK) return rc;
+    gleam_dims d = *dims;
+    d.workspace = scratch;
+    d.workspace_bytes = GLEAM_STATIC_SCRATCH_BYTES;
+    // Every scratch element that the kernels read is written earlier in the same call, so nothing
+    // has to be cleared between calls even though the array keeps the previous call's contents.
+    return gleam::run(x, y, sens, mask, eta, out, &d);
+}
+
 GLEAM_API uint64_t gleam_dc_launch_count(void) { return gleam::g_launches.load(); }
 
 GLEAM_API int gleam_dc_profile_begin(void) {

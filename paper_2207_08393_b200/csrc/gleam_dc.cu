@@ -64,6 +64,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     L->images = (long long)L->B * L->T;
     L->units = L->images * L->C;
     if (L->V > (1ll << 40) || L->units * L->V > (1ll << 46)) return GLEAM_ERR_BAD_DIMS;
+    if (L->images * L->n0 * L->n1 >= (1ll << 31)) return GLEAM_ERR_BAD_DIMS;   // row counters are 32-bit
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
     L->off_z = L->off_W = 0; L->G = 0;
@@ -152,7 +153,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
     const void* ptrs[6] = {x, y, sens, mask, out, d->workspace};
     for (int i = 0; i < 6; ++i) {
         if (!ptrs[i]) continue;
-        if (((uintptr_t)ptrs[i] & 7) != 0) return GLEAM_ERR_BAD_DIMS;
+        if (((uintptr_t)ptrs[i] & 15) != 0) return GLEAM_ERR_BAD_DIMS;   // 16-byte copies
         rc = check_device_ptr(ptrs[i]);
         if (rc != GLEAM_OK) return rc;
     }

@@ -2,6 +2,7 @@
 // unit that instantiates the kernels of that length.
 #pragma once
 #include "dc_kernels.cuh"
+#include "dc_warpline.cuh"
 
 namespace gleam {
 
@@ -34,6 +35,33 @@ inline cudaError_t launch_row(const RowArgs& a, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+// persistent launch of the warp-resident row kernel: one block per resident slot, warps stride
+// over the line groups
+template <class P, int MODE>
+inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
+    using WL = WarpLine<P, MODE>;
+    constexpr int WARPS = 1;
+    constexpr size_t SMEM = sizeof(cf) * WARPS * WL::WARP_ELEMS_ALIGNED;
+    static bool attr_done = false;
+    static int slots = 0;
+    cudaError_t e = ensure_smem(warpline_kernel<P, WARPS, MODE>, SMEM, attr_done);
+    if (e != cudaSuccess) return e;
+    if (slots == 0) {
+        int dev = 0, sms = 0, per_sm = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warpline_kernel<P, WARPS, MODE>, WARPS * 32,
+                                                               SMEM)) != cudaSuccess) return e;
+        slots = sms * (per_sm > 0 ? per_sm : 1);
+    }
+    const long long groups = (a.nrows + WL::LW - 1) / WL::LW;
+    long long blocks = (groups + WARPS - 1) / WARPS;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > slots) blocks = slots;
+    warpline_kernel<P, WARPS, MODE><<<(unsigned)blocks, WARPS * 32, SMEM, s>>>(a);
+    return cudaGetLastError();
+}
+
 template <class P, int L, int MODE>
 inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
     using E = LineFFT<P, true, L>;
@@ -50,11 +78,15 @@ inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
 
 template <class P, int LR, class PC, int LC>
 struct SizeImpl {
+    template <int MODE> static cudaError_t row_mode(const RowArgs& a, cudaStream_t s) {
+        if constexpr (WarpLine<P, MODE>::ELIGIBLE) return launch_warpline<P, MODE>(a, s);
+        else return launch_row<P, LR, MODE>(a, s);
+    }
     static cudaError_t row(int mode, const RowArgs& a, cudaStream_t s) {
         switch (mode) {
-            case ROW_FUSED: return launch_row<P, LR, ROW_FUSED>(a, s);
-            case ROW_FWD:   return launch_row<P, LR, ROW_FWD>(a, s);
-            case ROW_INV:   return launch_row<P, LR, ROW_INV>(a, s);
+            case ROW_FUSED: return row_mode<ROW_FUSED>(a, s);
+            case ROW_FWD:   return row_mode<ROW_FWD>(a, s);
+            case ROW_INV:   return row_mode<ROW_INV>(a, s);
         }
         return cudaErrorInvalidValue;
     }

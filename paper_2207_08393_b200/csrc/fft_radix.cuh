@@ -56,8 +56,30 @@ constexpr double sin2pi(long long k, long long n) {
 // ------------------------------------------------------------------------------------------
 // complex helpers
 // ------------------------------------------------------------------------------------------
-GLEAM_HD cf cadd(cf a, cf b) { return make_float2(a.x + b.x, a.y + b.y); }
-GLEAM_HD cf csub(cf a, cf b) { return make_float2(a.x - b.x, a.y - b.y); }
+// Complex add / subtract / real-scaled accumulate use the packed two-lane FP32 instructions of
+// sm_100 (one issue slot for both components); rounding is identical to the scalar forms.
+GLEAM_HD cf cadd(cf a, cf b) {
+#if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ >= 1000)
+    return __fadd2_rn(a, b);
+#else
+    return make_float2(a.x + b.x, a.y + b.y);
+#endif
+}
+GLEAM_HD cf csub(cf a, cf b) {
+#if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ >= 1000)
+    return __ffma2_rn(b, make_float2(-1.f, -1.f), a);
+#else
+    return make_float2(a.x - b.x, a.y - b.y);
+#endif
+}
+// acc + c * a  with a real constant c
+GLEAM_HD cf caxpy(float c, cf a, cf acc) {
+#if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ >= 1000)
+    return __ffma2_rn(make_float2(c, c), a, acc);
+#else
+    return make_float2(fmaf(c, a.x, acc.x), fmaf(c, a.y, acc.y));
+#endif
+}
 GLEAM_HD cf cmul(cf a, cf b) { return make_float2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x); }
 GLEAM_HD cf cmulc(cf a, cf b) { return make_float2(a.x * b.x + a.y * b.y, a.y * b.x - a.x * b.y); }  // a * conj(b)
 GLEAM_HD cf cscale(cf a, float s) { return make_float2(a.x * s, a.y * s); }
@@ -119,9 +141,16 @@ template <int DIR> struct Dft<2, DIR> {
 template <int DIR> struct Dft<4, DIR> {
     static GLEAM_HD void run(cf (&v)[4]) {
         const cf s02 = cadd(v[0], v[2]), d02 = csub(v[0], v[2]);
-        const cf s13 = cadd(v[1], v[3]), d13 = mul_i_dir<DIR>(csub(v[1], v[3]));
+        const cf s13 = cadd(v[1], v[3]), d13 = csub(v[1], v[3]);
         v[0] = cadd(s02, s13); v[2] = csub(s02, s13);
-        v[1] = cadd(d02, d13); v[3] = csub(d02, d13);
+        // v1 = d02 + (DIR i) d13,  v3 = d02 - (DIR i) d13   (component-wise: no register swap needed)
+        if (DIR > 0) {
+            v[1] = make_float2(d02.x - d13.y, d02.y + d13.x);
+            v[3] = make_float2(d02.x + d13.y, d02.y - d13.x);
+        } else {
+            v[1] = make_float2(d02.x + d13.y, d02.y - d13.x);
+            v[3] = make_float2(d02.x - d13.y, d02.y + d13.x);
+        }
     }
 };
 
@@ -146,13 +175,17 @@ template <int P, int DIR> struct DftPrime {
                 constexpr int m = decltype(mi)::value + 1;
                 constexpr float c = float(ct::cos2pi((long long)k * m, P));
                 constexpr float s = float(ct::sin2pi((long long)k * m, P));
-                C.x = fmaf(c, a[m - 1].x, C.x); C.y = fmaf(c, a[m - 1].y, C.y);
-                D.x = fmaf(s, b[m - 1].x, D.x); D.y = fmaf(s, b[m - 1].y, D.y);
+                C = caxpy(c, a[m - 1], C);
+                D = caxpy(s, b[m - 1], D);
             });
             // X[k] = C + DIR * i * D ,  X[P-k] = C - DIR * i * D
-            const cf iD = mul_i_dir<DIR>(D);
-            v[k] = cadd(C, iD);
-            v[P - k] = csub(C, iD);
+            if (DIR > 0) {
+                v[k] = make_float2(C.x - D.y, C.y + D.x);
+                v[P - k] = make_float2(C.x + D.y, C.y - D.x);
+            } else {
+                v[k] = make_float2(C.x + D.y, C.y - D.x);
+                v[P - k] = make_float2(C.x - D.y, C.y + D.x);
+            }
         });
     }
 };

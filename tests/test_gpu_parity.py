@@ -155,7 +155,7 @@ def test_error_codes_on_device_buffers():
         g.gleam_dc_forward(x, y, s, m, 1.0, y, d)               # out overlaps y
     assert e.value.status == binding.GLEAM_ERR_ALIAS
     with pytest.raises(g.GleamError) as e:
-        g.gleam_dc_vjp(x, s, m, 1.0, x.view(torch.float32)[..., 2:].data_ptr(), d)   # partial overlap
+        g.gleam_dc_vjp(x, s, m, 1.0, x.view(torch.float32)[..., 4:].data_ptr(), d)   # partial overlap
     assert e.value.status == binding.GLEAM_ERR_ALIAS
     g.gleam_dc_forward(x, y, s, m, 1.0, x, d)                  # exact alias is allowed
     torch.cuda.synchronize()

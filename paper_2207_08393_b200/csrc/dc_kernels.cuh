@@ -24,7 +24,8 @@ struct RowArgs {
     const cf* sens;     // (B,C,[T],n0,n1,n2)
     cf* out;            // (B,T,n0,n1,n2)
     const float* mask;  // ROW_FUSED: readout-invariant mask (B,T,n2)
-    const cf* z;        // ROW_FUSED: (B,C,T,n1,n2) shifted, signed, masked R^H y; may be null
+    const cf* z;        // ROW_FUSED: compact table of shifted, signed, masked R^H y: (B,C,T,n1,[rank < n2]); may be null
+    const int* zidx;    // fallback row kernel with z: (B,T,n2) rank of a raw k index among the sampled ones, -1 if unsampled
     cf* W;              // workspace (unit, rpb, n2)
     float eta;
     int C, T, Ts;       // coils, frames, sens frames (T or 1)
@@ -37,8 +38,11 @@ struct RowArgs {
 struct ColArgs {
     cf* W;              // in-place data (COL_MID_*, COL_FWD, COL_INV)
     const cf* y;        // COL_Z input / COL_MID_FULL measurements (B,C,T,V)
-    cf* z;              // COL_Z output
-    const cf* zin;      // COL_MID_SEP: z table (unit, n0, n1, n2)
+    cf* z;              // COL_Z output: compact table (unit, n_ro, [rank < pe])
+    const cf* zin;      // COL_MID_SEP: compact z table (unit, n0, [rank < n1 n2])
+    const int* zidx;    // (B,T,pe): rank of a raw k position among the sampled ones, -1 if unsampled
+    const int* zlist;   // (B,T,pe): sampled source positions p (unshifted), by rank
+    const int* zcount;  // (B,T)
     const float* mask;  // COL_Z, COL_MID_SEP: readout-invariant mask; COL_MID_FULL: full mask (B,T,V)
     int es;             // element stride of the transformed axis = lines per outer index
     long long nouter;   // outer indices
@@ -125,12 +129,17 @@ row_kernel(const RowArgs a) {
         }
     };
     load_s(s_cur, 0);
-    if (MODE == ROW_INV || use_z) load_k(k_cur, 0);
+    if (MODE == ROW_INV) load_k(k_cur, 0);
+    int zi[RL];
+    if (use_z && actL) {
+#pragma unroll
+        for (int k = 0; k < RL; ++k) zi[k] = a.zidx[btL * N + d.jL + P::BFL * k];
+    }
 
     for (int c = 0; c < a.C; ++c) {
         if (c + 1 < a.C) {
             load_s(s_nxt, c + 1);
-            if (MODE == ROW_INV || use_z) load_k(k_nxt, c + 1);
+            if (MODE == ROW_INV) load_k(k_nxt, c + 1);
         }
         cf v[R0], u[RL];
         if (MODE != ROW_INV) {
@@ -146,9 +155,15 @@ row_kernel(const RowArgs a) {
         if (MODE == ROW_FUSED) {
             if (actL) {
                 if (use_z) {
+                    const cf* zrow = a.z + (k_base - d.jL) + c * k_stride;
 #pragma unroll
-                    for (int k = 0; k < RL; ++k)
-                        u[k] = make_float2(fmaf(m2v[k], u[k].x, -k_cur[k].x), fmaf(m2v[k], u[k].y, -k_cur[k].y));
+                    for (int k = 0; k < RL; ++k) {
+                        u[k] = cscale(u[k], m2v[k]);
+                        if (zi[k] >= 0) {
+                            const cf q = zrow[zi[k]];
+                            u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
+                        }
+                    }
                 } else {
 #pragma unroll
                     for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], m2v[k]);
@@ -219,37 +234,37 @@ col_kernel(const ColArgs a) {
     cf v[R0], u[RL];
 
     if (MODE == COL_Z) {
-        // z = (g/sqrt(N_ro N_pe)) (-1)^{n_ro} (-1)^{p} M[p] * Rraw^H( (-1)^{k_ro} y ),  stored at sh(p)
-        // outer o = unit (b,c,t); inner i = phase-encode position p (flat over n1,n2 for rank 3)
+        // Lines are the sampled phase-encode positions of this unit's (b,t), by rank r.
+        // z[r] = (g/sqrt(N_ro N_pe)) (-1)^{n_ro} (-1)^{p} M[p] * Rraw^H( (-1)^{k_ro} y[.., p] ),  p = zlist[r]
         const int t = (int)(o % a.T);
         const int b = (int)(o / ((long long)a.C * a.T));
-        float mv = 0.f; int dest = 0, psign = 0;
-        if (line_ok) {
-            const long long pe = a.es;
-            mv = a.mask[((long long)b * a.T + t) * pe + i];
-            if (a.rank == 2) { dest = shift_half(i, a.n2); psign = i & 1; }
-            else {
-                const int i1 = i / a.n2, i2 = i % a.n2;
-                dest = shift_half(i1, a.n1) * a.n2 + shift_half(i2, a.n2);
-                psign = (i1 + i2) & 1;
-            }
+        const long long bt = (long long)b * a.T + t;
+        const long long pe = a.es;
+        const int cnt = a.zcount[bt];
+        if (i_base >= cnt) return;                      // whole block beyond the sampled set
+        const bool ok = i < cnt;
+        int p = 0, psign = 0; float mv = 0.f;
+        if (ok) {
+            p = a.zlist[bt * pe + i];
+            mv = a.mask[bt * pe + p];
+            psign = (a.rank == 2) ? (p & 1) : ((p / a.n2 + p % a.n2) & 1);
         }
-        if (actL) {
+        if (d.aL && ok) {
 #pragma unroll
             for (int k = 0; k < RL; ++k) {
                 const int kk = d.jL + P::BFL * k;
-                cf yv = (mv != 0.f) ? a.y[base + (long long)kk * a.es] : make_float2(0.f, 0.f);
+                const cf yv = a.y[o * (long long)N * pe + (long long)kk * pe + p];
                 u[k] = (kk & 1) ? make_float2(-yv.x, -yv.y) : yv;
             }
         }
         E::inverse(u, v, tw, d, smem);
-        if (act0) {
+        if (d.a0 && ok) {
             const float f = (psign ? -a.scale : a.scale) * mv;
 #pragma unroll
             for (int m = 0; m < R0; ++m) {
                 const int n = d.j0 + P::BF0 * m;
                 const float ff = (n & 1) ? -f : f;
-                a.z[o * (long long)N * a.es + (long long)n * a.es + dest] = cscale(v[m], ff);
+                a.z[o * (long long)N * pe + (long long)n * pe + i] = cscale(v[m], ff);
             }
         }
         return;
@@ -288,17 +303,17 @@ col_kernel(const ColArgs a) {
             const int b = (int)(unit / ((long long)a.C * a.T));
             const long long pe = (long long)a.n1 * a.n2;
             const float* mk = a.mask + ((long long)b * a.T + t) * pe + shift_half(i, a.n2);
-            const cf* zz = a.zin ? a.zin + (unit * a.n0 + a.i0_start + gi) * pe + i : nullptr;
+            const cf* zz = a.zin ? a.zin + (unit * a.n0 + a.i0_start + gi) * pe : nullptr;
+            const int* zi = a.zidx + ((long long)b * a.T + t) * pe + i;
 #pragma unroll
             for (int k = 0; k < RL; ++k) {
                 const long long kk = (long long)(d.jL + P::BFL * k) * a.n2;
                 const float mv = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
                 const float w = mv * mv * a.scale2;
-                if (zz) {
-                    const cf q = zz[kk];
-                    u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
-                } else {
-                    u[k] = cscale(u[k], w);
+                u[k] = cscale(u[k], w);
+                if (zz && mv != 0.f) {
+                    const cf q = zz[zi[kk]];
+                    u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
                 }
             }
         }

@@ -23,7 +23,7 @@ template <int NKEEP> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(NKEEP) : "memory");
 }
 
-template <class P, int MODE>
+template <class P, int MODE, bool HAS_Z = false>
 struct WarpLine {
     static constexpr int N = P::N, R0 = P::R0, RL = P::RL, S = P::S;
     static constexpr int BFMAX = cmax(P::BF0, P::BFL);
@@ -33,18 +33,25 @@ struct WarpLine {
     static constexpr int EXL = (S == 2) ? P::SM_A : 0;    // exchange elements per line
     // per-warp shared memory, in float2 units: S[2], K[2] (z or W; not in ROW_FWD), x (not in
     // ROW_INV), exchange, m2 (ROW_FUSED; floats, N/2 float2 per line)
+    // K stage: a whole line of the workspace (ROW_INV), or up to KCAP sampled z entries per line
+    // (ROW_FUSED with z; lines with more sampled positions read z straight from global memory).
     static constexpr int TILE = LW * N;
-    static constexpr bool HAS_K = (MODE != ROW_FWD), HAS_X = (MODE != ROW_INV), HAS_M = (MODE == ROW_FUSED);
-    static constexpr int OFF_S = 0, OFF_K = 2 * TILE, OFF_X = OFF_K + (HAS_K ? 2 * TILE : 0),
+    static constexpr int KCAP = (MODE == ROW_INV) ? N : (((N + 3) / 4 + 1) / 2 * 2);
+    static constexpr int KTILE = LW * KCAP;
+    static constexpr bool HAS_K = (MODE == ROW_INV) || (MODE == ROW_FUSED && HAS_Z);
+    static constexpr bool HAS_X = (MODE != ROW_INV), HAS_M = (MODE == ROW_FUSED), HAS_I = (MODE == ROW_FUSED && HAS_Z);
+    static constexpr int OFF_S = 0, OFF_K = 2 * TILE, OFF_X = OFF_K + (HAS_K ? 2 * KTILE : 0),
                          OFF_EX = OFF_X + (HAS_X ? TILE : 0), OFF_M2 = OFF_EX + LW * EXL + (LW * EXL) % 2;
-    static constexpr int WARP_ELEMS = OFF_M2 + (HAS_M ? TILE / 2 : 0) + 2;
+    static constexpr int OFF_IDX = OFF_M2 + (HAS_M ? TILE / 2 : 0);     // ranks of the raw k indices (ints)
+    static constexpr int WARP_ELEMS = OFF_IDX + (HAS_I ? TILE / 2 : 0) + 2;
     static constexpr int WARP_ELEMS_ALIGNED = (WARP_ELEMS + 1) / 2 * 2;   // keep 16-byte alignment per warp
 };
 
-template <class P, int WARPS, int MODE>
+template <class P, int WARPS, int MODE, bool HAS_Z>
 __global__ void __launch_bounds__(WARPS * 32)
 warpline_kernel(const RowArgs a) {
-    using WL = WarpLine<P, MODE>;
+    using WL = WarpLine<P, MODE, HAS_Z>;
+    constexpr int KCAP = WL::KCAP, KTILE = WL::KTILE;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL, TPL = WL::TPL, LW = WL::LW, TILE = WL::TILE;
     extern __shared__ __align__(16) float2 smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -54,6 +61,7 @@ warpline_kernel(const RowArgs a) {
     cf* sX = wsm + WL::OFF_X;
     cf* sE = wsm + WL::OFF_EX;
     float* sM = reinterpret_cast<float*>(wsm + WL::OFF_M2);
+    int* sI = reinterpret_cast<int*>(wsm + WL::OFF_IDX);
 
     const int l = lane / TPL, j = lane % TPL;
     const bool a0 = j < P::BF0, aL = j < P::BFL;
@@ -66,8 +74,8 @@ warpline_kernel(const RowArgs a) {
 
     const long long ngroups = (a.nrows + LW - 1) / LW;
     const long long wstride = (long long)gridDim.x * WARPS;
-    const bool use_z = (MODE == ROW_FUSED) && (a.z != nullptr);
-    const bool use_k = (MODE == ROW_INV) || use_z;
+    constexpr bool use_z = (MODE == ROW_FUSED) && HAS_Z;
+    constexpr bool use_k = (MODE == ROW_INV) || use_z;
 
     for (long long g = (long long)blockIdx.x * WARPS + warp; g < ngroups; g += wstride) {
         // ---- element offsets of this lane's line; other lines' offsets come by shuffle ----
@@ -84,18 +92,23 @@ warpline_kernel(const RowArgs a) {
         const long long s_stride = (long long)a.Ts * a.RPB * N;
         const long long k_stride = (long long)a.T * ((MODE == ROW_FUSED) ? a.RPB : a.rpb) * N;
 
+        // entries of this line's K row to stage: the whole row (ROW_INV) or the number of sampled
+        // positions (z; set below, when the mask row is scanned)
+        int k_cnt = (MODE == ROW_INV) ? N : 0;
+
         auto issue_coil = [&](int c, int buf) {
 #pragma unroll
             for (int ll = 0; ll < LW; ++ll) {
                 const bool ok = __shfl_sync(0xffffffffu, (int)row_ok, ll * TPL) != 0;
                 const long long so = __shfl_sync(0xffffffffu, s_off, ll * TPL);
                 const long long ko = __shfl_sync(0xffffffffu, k_off, ll * TPL);
+                const int kc = __shfl_sync(0xffffffffu, k_cnt, ll * TPL);
                 if (!ok) continue;
                 const cf* src = a.sens + so + c * s_stride;
                 for (int i = lane; i < N / 2; i += 32) cp_async16(sS + buf * TILE + ll * N + 2 * i, src + 2 * i);
-                if (use_k) {
+                if (use_k && kc <= KCAP) {
                     const cf* ks = ((MODE == ROW_FUSED) ? a.z : a.W) + ko + c * k_stride;
-                    for (int i = lane; i < N / 2; i += 32) cp_async16(sK + buf * TILE + ll * N + 2 * i, ks + 2 * i);
+                    for (int i = lane; i < (kc + 1) / 2; i += 32) cp_async16(sK + buf * KTILE + ll * KCAP + 2 * i, ks + 2 * i);
                 }
             }
         };
@@ -111,10 +124,20 @@ warpline_kernel(const RowArgs a) {
                 for (int i = lane; i < N / 2; i += 32) cp_async16(sX + ll * N + 2 * i, a.x + xo + 2 * i);
             }
             if (MODE == ROW_FUSED) {
-                for (int k = lane; k < N; k += 32) {
-                    const float mv = a.mask[bto * N + shift_half(k, N)];
-                    sM[ll * N + k] = mv * mv * (1.0f / N);
+                // scaled mask^2 in raw k order and, with z, the rank of every sampled k (the order
+                // in which the z table was written)
+                int cnt = 0;
+                for (int k0 = 0; k0 < N; k0 += 32) {
+                    const int k = k0 + lane;
+                    const float mv = (k < N) ? a.mask[bto * N + shift_half(k, N)] : 0.f;
+                    if (k < N) sM[ll * N + k] = mv * mv * (1.0f / N);
+                    if (use_z) {
+                        const unsigned bal = __ballot_sync(0xffffffffu, mv != 0.f);
+                        if (k < N) sI[ll * N + k] = (mv != 0.f) ? cnt + __popc(bal & ((1u << lane) - 1u)) : -1;
+                        cnt += __popc(bal);
+                    }
                 }
+                if (use_z && l == ll) k_cnt = cnt;
             }
         }
         issue_coil(0, 0);
@@ -132,7 +155,8 @@ warpline_kernel(const RowArgs a) {
             __syncwarp();
 
             const cf* cS = sS + buf * TILE + l * N;
-            const cf* cK = sK + buf * TILE + l * N;
+            const cf* cK = sK + buf * KTILE + l * KCAP;
+            const cf* gK = use_z ? a.z + k_off + c * k_stride : nullptr;   // this line's compact z row
             const cf* cX = sX + l * N;
             cf v[R0], u[RL];
             if (MODE != ROW_INV) {
@@ -165,11 +189,13 @@ warpline_kernel(const RowArgs a) {
 #pragma unroll
                     for (int k = 0; k < RL; ++k) {
                         const float w = mm[j + P::BFL * k];
-                        if (use_z) {
-                            const cf q = cK[j + P::BFL * k];
-                            u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
-                        } else {
-                            u[k] = cscale(u[k], w);
+                        u[k] = cscale(u[k], w);
+                        if (use_z && row_ok) {      // lanes without a row hold no rank table
+                            const int r = sI[l * N + j + P::BFL * k];
+                            if (r >= 0 && r < N) {
+                                const cf q = (k_cnt <= KCAP) ? cK[r] : gK[r];
+                                u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
+                            }
                         }
                     }
                 }

@@ -3,7 +3,7 @@
 
 namespace gleam {
 #define GLEAM_SIZE(N, A0, A1, A2, LR, B0, B1, B2, LC) \
-    extern const SizeOps size_ops_##N = {N, &SizeImpl<Plan<N, A0, A1, A2>, LR, Plan<N, B0, B1, B2>, LC>::row, \
+    extern const SizeOps size_ops_##N = {N, WarpLine<Plan<N, A0, A1, A2>, ROW_FUSED>::ELIGIBLE, &SizeImpl<Plan<N, A0, A1, A2>, LR, Plan<N, B0, B1, B2>, LC>::row, \
                                          &SizeImpl<Plan<N, A0, A1, A2>, LR, Plan<N, B0, B1, B2>, LC>::col};
 #include "sizes.def"
 #undef GLEAM_SIZE

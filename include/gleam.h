@@ -166,7 +166,7 @@ GLEAM_API uint64_t gleam_dc_static_scratch_bytes(void);
  * Profiling creates CUDA events on first use and is meant for benchmarks, not for production.
  */
 enum {
-    GLEAM_K_PREP_M2 = 0,      /* mask table */
+    GLEAM_K_PREP_M2 = 0,      /* rank map of the sampled positions (forward call only) */
     GLEAM_K_COL_Z = 1,        /* readout-axis inverse transform of y */
     GLEAM_K_ROW_FUSED = 2,    /* 2-D one-pass kernel */
     GLEAM_K_ROW_FWD = 3,      /* sensitivity multiply + transform of the contiguous axis */

@@ -34,6 +34,65 @@ static const SizeOps* find_size(int n) {
     }
 }
 
+// Ranks of the sampled phase-encode positions, in the order of the raw (half-shifted) k index q:
+//   zidx[bt][q]  = rank of q among the sampled positions, or -1 where M[sh(q)] == 0
+//   zlist[bt][r] = unshifted source position p = sh(q) of rank r;   zcount[bt] = number sampled.
+// Block (chunk, bt) owns ZMAP_CHUNK consecutive q; it counts the sampled positions before its chunk
+// by itself (no communication between blocks), then scans its own chunk.
+#define ZMAP_THREADS 256
+#define ZMAP_PER_THREAD 8
+#define ZMAP_CHUNK (ZMAP_THREADS * ZMAP_PER_THREAD)
+__global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restrict__ mask, int* __restrict__ zidx,
+                                                            int* __restrict__ zlist, int* __restrict__ zcount,
+                                                            int n1, int n2, int rank) {
+    __shared__ int warp_sum[ZMAP_THREADS / 32];
+    __shared__ int base_sh;
+    const int pe = (rank == 2) ? n2 : n1 * n2;
+    const long long bt = blockIdx.y;
+    const float* mk = mask + bt * pe;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q_begin = blockIdx.x * ZMAP_CHUNK;
+    auto src_of = [&](int q) -> int {
+        if (rank == 2) return shift_half(q, n2);
+        return shift_half(q / n2, n1) * n2 + shift_half(q % n2, n2);
+    };
+    // sampled positions before this chunk
+    int c = 0;
+    for (int q = tid; q < q_begin; q += ZMAP_THREADS) c += (mk[src_of(q)] != 0.f) ? 1 : 0;
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if (lane == 0) warp_sum[warp] = c;
+    __syncthreads();
+    if (tid == 0) { int t = 0; for (int w = 0; w < ZMAP_THREADS / 32; ++w) t += warp_sum[w]; base_sh = t; }
+    __syncthreads();
+    const int base = base_sh;
+    __syncthreads();
+    // this chunk: each thread owns ZMAP_PER_THREAD consecutive q
+    const int q0 = q_begin + tid * ZMAP_PER_THREAD;
+    int src[ZMAP_PER_THREAD]; bool on[ZMAP_PER_THREAD]; int mine = 0;
+#pragma unroll
+    for (int e = 0; e < ZMAP_PER_THREAD; ++e) {
+        const int q = q0 + e;
+        src[e] = (q < pe) ? src_of(q) : 0;
+        on[e] = (q < pe) && (mk[src[e]] != 0.f);
+        mine += on[e] ? 1 : 0;
+    }
+    int incl = mine;                                         // inclusive scan inside the warp
+    for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    int wbase = 0;
+    for (int w = 0; w < warp; ++w) wbase += warp_sum[w];
+    int r = base + wbase + incl - mine;
+#pragma unroll
+    for (int e = 0; e < ZMAP_PER_THREAD; ++e) {
+        const int q = q0 + e;
+        if (q >= pe) break;
+        if (on[e]) { zidx[bt * pe + q] = r; zlist[bt * pe + r] = src[e]; ++r; }
+        else zidx[bt * pe + q] = -1;
+    }
+    if (q_begin + ZMAP_CHUNK >= pe && tid == ZMAP_THREADS - 1) zcount[bt] = r;   // last chunk, last thread: total
+}
+
 static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
@@ -42,7 +101,7 @@ struct Layout {
     long long V, units, images;
     bool separable;
     // workspace (byte offsets)
-    uint64_t off_z, off_W, total;
+    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_W, total;
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
@@ -64,13 +123,20 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     L->images = (long long)L->B * L->T;
     L->units = L->images * L->C;
     if (L->V > (1ll << 40) || L->units * L->V > (1ll << 46)) return GLEAM_ERR_BAD_DIMS;
+    if ((long long)L->n1 * L->n2 >= (1ll << 30) || L->images > 65535) return GLEAM_ERR_BAD_DIMS;   // rank map: 32-bit positions, grid.y
     if (L->images * L->n0 * L->n1 >= (1ll << 31)) return GLEAM_ERR_BAD_DIMS;   // row counters are 32-bit
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
-    L->off_z = L->off_W = 0; L->G = 0;
+    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_W = 0; L->G = 0;
     if (L->separable) {
         const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
-        if (with_y) { L->off_z = off; off = align_up(off + (uint64_t)L->units * L->V * sizeof(cf), 256); }
+        if (with_y) {
+            // compact z table, sized for the worst case (every position sampled), and the rank maps
+            L->off_z = off; off = align_up(off + (uint64_t)L->units * L->V * sizeof(cf), 256);
+            L->off_zidx = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(int), 256);
+            L->off_zlist = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(int), 256);
+            L->off_zcount = off; off = align_up(off + (uint64_t)L->images * sizeof(int), 256);
+        }
         if (L->rank == 3) {
             const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
             long long G = (long long)(CHUNK_TARGET_BYTES / slab);
@@ -184,7 +250,17 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
     if (L.separable) {
         cf* z = y ? (cf*)(ws + L.off_z) : nullptr;
         if (y) {
-            // z table: inverse transform of y along the readout axis, at sampled positions
+            // ranks of the sampled positions, then the z table: inverse transform of y along the
+            // readout axis at the sampled positions only
+            int* zidx = (int*)(ws + L.off_zidx);
+            int* zlist = (int*)(ws + L.off_zlist);
+            int* zcount = (int*)(ws + L.off_zcount);
+            CK(prof_mark(GLEAM_K_PREP_M2, s));
+            zmap_kernel<<<dim3((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images), ZMAP_THREADS, 0, s>>>(
+                mask, zidx, zlist, zcount, L.n1, L.n2, L.rank);
+            CK(cudaGetLastError());
+            ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount;
+            ra.zidx = zidx;
             ColArgs cz = ca;
             cz.y = (const cf*)y; cz.z = z; cz.mask = mask;
             cz.es = (int)pe; cz.nouter = L.units;

@@ -1,0 +1,113 @@
+// Pipelined variant of col_kernel<COL_MID_SEP> (strided-axis transform, mask + residual, inverse,
+// in place on the workspace chunk) for two-stage plans.
+//
+// A block is persistent: it walks over tiles of L neighbouring strided lines and, while it
+// transforms one tile, the next one streams from the (L2-resident) workspace into shared memory
+// with cp.async.  Three shared-memory buffers rotate between the roles "incoming tile",
+// "forward exchange" (the buffer the current tile arrived in, once every thread holds its
+// elements in registers) and "inverse exchange".
+#pragma once
+#include "dc_warpline.cuh"
+
+namespace gleam {
+
+template <class P, int L>
+struct ColPipe {
+    static constexpr bool ELIGIBLE = (P::S == 2) && (L % 2 == 0);
+    static constexpr int BUFSZ = L * cmax(P::BUF, P::N);            // elements per buffer
+    static constexpr size_t SMEM_BYTES = sizeof(cf) * (3 * BUFSZ + 2);
+    static constexpr int THREADS = LineFFT<P, true, L>::THREADS;
+};
+
+template <class P, int L>
+__global__ void __launch_bounds__(ColPipe<P, L>::THREADS)
+colpipe_mid_sep_kernel(const ColArgs a) {
+    using E = LineFFT<P, true, L>;
+    using CP = ColPipe<P, L>;
+    constexpr int N = P::N, R0 = P::R0, RL = P::RL;
+    extern __shared__ __align__(16) float2 smem[];
+    cf* buf[3] = {smem, smem + CP::BUFSZ, smem + 2 * CP::BUFSZ};
+    const typename E::Ids d = E::ids(threadIdx.x);
+    typename E::Tw tw;
+    E::make_tw(d, tw);
+
+    const int tiles_per_o = (a.es + L - 1) / L;
+    const long long ntiles = a.nouter * tiles_per_o;
+    const long long pe = (long long)a.n1 * a.n2;
+
+    // stream tile `tile` into `dst` in [n][l] layout; chunks of 16 bytes (two neighbouring lines)
+    auto issue = [&](long long tile, cf* dst) {
+        const long long o = tile / tiles_per_o;
+        const int i_base = (int)(tile - o * tiles_per_o) * L;
+        const cf* src = a.W + o * (long long)N * a.es + i_base;
+        for (int c = threadIdx.x; c < N * (L / 2); c += CP::THREADS) {
+            const int n = c / (L / 2), part = c - n * (L / 2);
+            if (i_base + 2 * part < a.es) cp_async16(dst + n * L + 2 * part, src + (long long)n * a.es + 2 * part);
+        }
+    };
+
+    long long tile = blockIdx.x;
+    if (tile < ntiles) issue(tile, buf[0]);
+    cp_async_commit();
+    int it = 0;
+    for (; tile < ntiles; tile += gridDim.x, ++it) {
+        cf* cur = buf[it % 3];
+        cf* nxt = buf[(it + 1) % 3];
+        cf* spare = buf[(it + 2) % 3];
+        cp_async_wait<0>();
+        __syncthreads();          // tile is visible to all; every thread has left the previous tile
+        if (tile + gridDim.x < ntiles) issue(tile + gridDim.x, nxt);
+        cp_async_commit();
+
+        const long long o = tile / tiles_per_o;
+        const int i_base = (int)(tile - o * tiles_per_o) * L;
+        const int i = i_base + d.l0;
+        const bool line_ok = i < a.es;
+        const bool act0 = d.a0 && line_ok, actL = d.aL && line_ok;
+        const long long base = o * (long long)N * a.es + i;
+        // chunk geometry: o = unit * G + gi
+        const long long unit = o / a.G;
+        const int gi = (int)(o - unit * a.G);
+        const int t = (int)(unit % a.T);
+        const int b = (int)(unit / ((long long)a.C * a.T));
+        const long long bt = (long long)b * a.T + t;
+
+        cf v[R0], u[RL];
+        float mw[RL];
+        if (act0) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) v[m] = cur[(d.j0 + P::BF0 * m) * L + d.l0];
+        } else {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) v[m] = make_float2(0.f, 0.f);
+        }
+        if (actL) {   // mask weights of this thread's k-space entries, issued early
+            const float* mk = a.mask + bt * pe + shift_half(i, a.n2);
+#pragma unroll
+            for (int k = 0; k < RL; ++k) mw[k] = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
+        }
+        __syncthreads();          // all elements are in registers: `cur` becomes the forward exchange
+        E::forward_xy(v, u, tw, d, cur, cur);
+        if (actL) {
+            const cf* zz = a.zin ? a.zin + (unit * a.n0 + a.i0_start + gi) * pe : nullptr;
+            const int* zi = a.zidx + bt * pe + i;
+#pragma unroll
+            for (int k = 0; k < RL; ++k) {
+                const float w = mw[k] * mw[k] * a.scale2;
+                u[k] = cscale(u[k], w);
+                if (zz && mw[k] != 0.f) {
+                    const cf q = zz[zi[(long long)(d.jL + P::BFL * k) * a.n2]];
+                    u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
+                }
+            }
+        }
+        E::inverse_xy(u, v, tw, d, spare, spare);
+        if (act0) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) a.W[base + (long long)(d.j0 + P::BF0 * m) * a.es] = v[m];
+        }
+    }
+    cp_async_wait<0>();
+}
+
+}  // namespace gleam

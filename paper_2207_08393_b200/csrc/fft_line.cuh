@@ -98,14 +98,19 @@ struct LineFFT {
     // call, the buffer written now must not be the one other threads may still be reading.
     __device__ __forceinline__ static void forward(cf (&v)[R0], cf (&u)[RL], const Tw& tw, const Ids& d, cf* sm,
                                                    int flip = 0) {
+        cf* X = sm + ((S == 2 && flip) ? (COL ? L * P::BUF : P::BUF) : 0);
+        cf* Y = sm + (COL ? L * P::BUF : P::BUF);
+        forward_xy(v, u, tw, d, X, Y);
+    }
+    // forward with explicit exchange buffers (two-stage plans use X only)
+    __device__ __forceinline__ static void forward_xy(cf (&v)[R0], cf (&u)[RL], const Tw& tw, const Ids& d, cf* X,
+                                                      cf* Y) {
         if (S == 1) {
             Dft<R0, -1>::run(v);
 #pragma unroll
             for (int k = 0; k < RL; ++k) u[k] = v[k % R0];
             return;
         }
-        cf* X = sm + ((S == 2 && flip) ? (COL ? L * P::BUF : P::BUF) : 0);
-        cf* Y = sm + (COL ? L * P::BUF : P::BUF);
         if (d.a0) {
             Dft<R0, -1>::run(v);
 #pragma unroll
@@ -148,14 +153,19 @@ struct LineFFT {
     // three-stage plans go through X then Y.
     __device__ __forceinline__ static void inverse(cf (&u)[RL], cf (&v)[R0], const Tw& tw, const Ids& d, cf* sm,
                                                    int flip = 0) {
+        cf* X = sm;
+        cf* Y = sm + ((S == 2 && flip) ? 0 : (COL ? L * P::BUF : P::BUF));
+        inverse_xy(u, v, tw, d, X, Y);
+    }
+    // inverse with explicit exchange buffers (two-stage plans use Y only)
+    __device__ __forceinline__ static void inverse_xy(cf (&u)[RL], cf (&v)[R0], const Tw& tw, const Ids& d, cf* X,
+                                                      cf* Y) {
         if (S == 1) {
 #pragma unroll
             for (int k = 0; k < R0; ++k) v[k] = u[k % RL];
             Dft<R0, +1>::run(v);
             return;
         }
-        cf* X = sm;
-        cf* Y = sm + ((S == 2 && flip) ? 0 : (COL ? L * P::BUF : P::BUF));
         if (S == 3) {
             if (d.aL) {
                 Dft<RL, +1>::run(u);

@@ -3,6 +3,7 @@
 #pragma once
 #include "dc_kernels.cuh"
 #include "dc_warpline.cuh"
+#include "dc_colpipe.cuh"
 
 namespace gleam {
 
@@ -83,6 +84,29 @@ inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+// persistent launch of the pipelined column kernel (separable 3-D path)
+template <class P, int L>
+inline cudaError_t launch_colpipe(const ColArgs& a, cudaStream_t s) {
+    using CP = ColPipe<P, L>;
+    static bool attr_done = false;
+    static int slots = 0;
+    cudaError_t e = ensure_smem(colpipe_mid_sep_kernel<P, L>, CP::SMEM_BYTES, attr_done);
+    if (e != cudaSuccess) return e;
+    if (slots == 0) {
+        int dev = 0, sms = 0, per_sm = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, colpipe_mid_sep_kernel<P, L>, CP::THREADS,
+                                                               CP::SMEM_BYTES)) != cudaSuccess) return e;
+        slots = sms * (per_sm > 0 ? per_sm : 1);
+    }
+    const long long tiles = a.nouter * ((a.es + L - 1) / L);
+    if (tiles <= 0) return cudaSuccess;
+    const long long blocks = tiles < slots ? tiles : slots;
+    colpipe_mid_sep_kernel<P, L><<<(unsigned)blocks, CP::THREADS, CP::SMEM_BYTES, s>>>(a);
+    return cudaGetLastError();
+}
+
 template <class P, int LR, class PC, int LC>
 struct SizeImpl {
     template <int MODE> static cudaError_t row_mode(const RowArgs& a, cudaStream_t s) {
@@ -100,7 +124,9 @@ struct SizeImpl {
     static cudaError_t col(int mode, const ColArgs& a, cudaStream_t s) {
         switch (mode) {
             case COL_Z:        return launch_col<PC, LC, COL_Z>(a, s);
-            case COL_MID_SEP:  return launch_col<PC, LC, COL_MID_SEP>(a, s);
+            case COL_MID_SEP:
+                if constexpr (ColPipe<PC, LC>::ELIGIBLE) return launch_colpipe<PC, LC>(a, s);
+                else return launch_col<PC, LC, COL_MID_SEP>(a, s);
             case COL_MID_FULL: return launch_col<PC, LC, COL_MID_FULL>(a, s);
             case COL_FWD:      return launch_col<PC, LC, COL_FWD>(a, s);
             case COL_INV:      return launch_col<PC, LC, COL_INV>(a, s);

@@ -20,7 +20,7 @@ struct ColPipe {
 };
 
 template <class P, int L>
-__global__ void __launch_bounds__(ColPipe<P, L>::THREADS)
+__global__ void __launch_bounds__(ColPipe<P, L>::THREADS, 3)
 colpipe_mid_sep_kernel(const ColArgs a) {
     using E = LineFFT<P, true, L>;
     using CP = ColPipe<P, L>;

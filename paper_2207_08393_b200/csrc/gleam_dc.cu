@@ -105,7 +105,17 @@ struct Layout {
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
-static const uint64_t CHUNK_TARGET_BYTES = 48ull << 20;   // keep the chunk workspace inside L2
+// Target size of the 3-D chunk workspace: it has to stay inside L2 between the three kernels of a
+// chunk.  GLEAM_CHUNK_MB overrides the default (tuning aid, read once).
+static uint64_t chunk_target_bytes() {
+    static uint64_t v = 0;
+    if (v == 0) {
+        const char* e = getenv("GLEAM_CHUNK_MB");
+        long mb = e ? atol(e) : 0;
+        v = (uint64_t)((mb > 0 && mb <= 4096) ? mb : 48) << 20;
+    }
+    return v;
+}
 
 static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     if (d->struct_version != GLEAM_DIMS_VERSION) return GLEAM_ERR_BAD_DIMS;
@@ -139,7 +149,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
         }
         if (L->rank == 3) {
             const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
-            long long G = (long long)(CHUNK_TARGET_BYTES / slab);
+            long long G = (long long)(chunk_target_bytes() / slab);
             if (G < 1) G = 1;
             if (G > L->n0) G = L->n0;
             L->G = (int)G;

@@ -90,7 +90,7 @@ def kernel_work(cls, w, launches_per_call):
 
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -104,8 +104,11 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples taken between the wall-clock times t_begin and t_end (the timed
+        region); if the region was too short to catch one, of all samples of the run under load."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "timed region"}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -116,6 +119,19 @@ class ClockSampler:
         self.tmp.flush()
         rows = [r.strip().split(",") for r in open(self.tmp.name) if r.strip()]
         os.unlink(self.tmp.name)
+
+        def stamp(r):
+            try:
+                return datetime.datetime.strptime(r[0].strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+            except ValueError:
+                return None
+        if t_begin is not None:
+            inside = [r[1:] for r in rows if (stamp(r) is not None and t_begin - 0.05 <= stamp(r) <= t_end + 0.05)]
+            if inside:
+                rows = [[None] + r for r in inside]
+            else:
+                out["window"] = "whole run (timed region shorter than the sampling interval)"
+        rows = [r[1:] for r in rows]
         sm, names = [], ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = set()
         for r in rows:
@@ -159,7 +175,7 @@ def reference_sample(w):
     """Bounded sample of a workload for the CPU oracle: same kind of problem, fewer units."""
     from paper_2207_08393_b200 import workloads as wl
     if w.name == "knee3d":
-        return wl.scaled(w, coils=2, n=(32, w.n[1], w.n[2])), "2 of 8 coils, 32 of 320 readout slabs (32x320x256)"
+        return wl.scaled(w, n=(16, w.n[1], w.n[2])), "8 coils, 16 of 320 readout slabs (16x320x256)"
     if w.name in ("knee2d", "brain2d"):
         return wl.scaled(w, batch=1), "batch 1 of %d" % w.batch
     return w, "whole workload"
@@ -246,13 +262,15 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3 if sampler else 0.0)       # let the sampler start before the GPU gets busy
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
 
     # ---- device-resident timed region -------------------------------------------------------
-    sampler = ClockSampler(local) if rank == 0 else None
     launches0 = g.gleam_dc_launch_count()
+    t_begin = time.time()
     if flush is None:
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
@@ -274,7 +292,7 @@ def run_ours(args, w):
         barrier()
         local_ms = sum(a.elapsed_time(b) for a, b in evs)
     launches = g.gleam_dc_launch_count() - launches0
-    clocks = sampler.stop() if sampler else None
+    t_end = time.time()
     total_ms, total_units = aggregate(local_ms, w.voxel_coils * args.steps, world, dist, dev)
     value = total_units / (total_ms * 1e-3)
 
@@ -304,6 +322,8 @@ def run_ours(args, w):
         ef[2].record(stream); torch.cuda.synchronize()
         split[0] += ef[0].elapsed_time(ef[1]) / prof_steps
         split[1] += ef[1].elapsed_time(ef[2]) / prof_steps
+
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
 
     # ---- end to end through the host-buffer entry points --------------------------------------
     e2e_steps = max(1, min(args.steps, 3 if inputs_bytes > (1 << 30) else 10))

@@ -31,13 +31,14 @@ colpipe_mid_sep_kernel(const ColArgs a) {
     typename E::Tw tw;
     E::make_tw(d, tw);
 
-    const int tiles_per_o = (a.es + L - 1) / L;
-    const long long ntiles = a.nouter * tiles_per_o;
+    // tile counters are 32-bit (the launcher refuses more than 2^31 tiles): no 64-bit divisions
+    const unsigned tiles_per_o = (unsigned)((a.es + L - 1) / L);
+    const unsigned ntiles = (unsigned)a.nouter * tiles_per_o;
     const long long pe = (long long)a.n1 * a.n2;
 
     // stream tile `tile` into `dst` in [n][l] layout; chunks of 16 bytes (two neighbouring lines)
-    auto issue = [&](long long tile, cf* dst) {
-        const long long o = tile / tiles_per_o;
+    auto issue = [&](unsigned tile, cf* dst) {
+        const unsigned o = tile / tiles_per_o;
         const int i_base = (int)(tile - o * tiles_per_o) * L;
         const cf* src = a.W + o * (long long)N * a.es + i_base;
         for (int c = threadIdx.x; c < N * (L / 2); c += CP::THREADS) {
@@ -46,7 +47,7 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         }
     };
 
-    long long tile = blockIdx.x;
+    unsigned tile = blockIdx.x;
     if (tile < ntiles) issue(tile, buf[0]);
     cp_async_commit();
     int it = 0;
@@ -59,17 +60,18 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         if (tile + gridDim.x < ntiles) issue(tile + gridDim.x, nxt);
         cp_async_commit();
 
-        const long long o = tile / tiles_per_o;
+        const unsigned o = tile / tiles_per_o;
         const int i_base = (int)(tile - o * tiles_per_o) * L;
         const int i = i_base + d.l0;
         const bool line_ok = i < a.es;
         const bool act0 = d.a0 && line_ok, actL = d.aL && line_ok;
         const long long base = o * (long long)N * a.es + i;
         // chunk geometry: o = unit * G + gi
-        const long long unit = o / a.G;
-        const int gi = (int)(o - unit * a.G);
-        const int t = (int)(unit % a.T);
-        const int b = (int)(unit / ((long long)a.C * a.T));
+        const unsigned unit = o / (unsigned)a.G;
+        const int gi = (int)(o - unit * (unsigned)a.G);
+        const unsigned bc = unit / (unsigned)a.T;
+        const int t = (int)(unit - bc * (unsigned)a.T);
+        const int b = (int)(bc / (unsigned)a.C);
         const long long bt = (long long)b * a.T + t;
 
         cf v[R0], u[RL];
@@ -89,7 +91,7 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         __syncthreads();          // all elements are in registers: `cur` becomes the forward exchange
         E::forward_xy(v, u, tw, d, cur, cur);
         if (actL) {
-            const cf* zz = a.zin ? a.zin + (unit * a.n0 + a.i0_start + gi) * pe : nullptr;
+            const cf* zz = a.zin ? a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe : nullptr;
             const int* zi = a.zidx + bt * pe + i;
 #pragma unroll
             for (int k = 0; k < RL; ++k) {

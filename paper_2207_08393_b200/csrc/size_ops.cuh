@@ -102,6 +102,7 @@ inline cudaError_t launch_colpipe(const ColArgs& a, cudaStream_t s) {
     }
     const long long tiles = a.nouter * ((a.es + L - 1) / L);
     if (tiles <= 0) return cudaSuccess;
+    if (tiles >= 2147483647LL) return cudaErrorInvalidConfiguration;
     const long long blocks = tiles < slots ? tiles : slots;
     colpipe_mid_sep_kernel<P, L><<<(unsigned)blocks, CP::THREADS, CP::SMEM_BYTES, s>>>(a);
     return cudaGetLastError();

@@ -144,6 +144,11 @@ warpline_kernel(const RowArgs a) {
         cp_async_commit();
 
         cf acc[R0];
+        cf xreg[R0];     // ROW_INV: x is needed only for the final update; fetched early, held in registers
+        if (!WL::HAS_X && a0 && row_ok) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) xreg[m] = a.x[x_off + j + P::BF0 * m];
+        }
 #pragma unroll
         for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
 
@@ -247,7 +252,7 @@ warpline_kernel(const RowArgs a) {
             if (a0 && row_ok) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
-                    const cf xv = WL::HAS_X ? sX[l * N + j + P::BF0 * m] : a.x[x_off + j + P::BF0 * m];
+                    const cf xv = WL::HAS_X ? sX[l * N + j + P::BF0 * m] : xreg[m];
                     a.out[x_off + j + P::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
                 }
             }

@@ -39,8 +39,8 @@ static const SizeOps* find_size(int n) {
 //   zlist[bt][r] = unshifted source position p = sh(q) of rank r;   zcount[bt] = number sampled.
 // Block (chunk, bt) owns ZMAP_CHUNK consecutive q; it counts the sampled positions before its chunk
 // by itself (no communication between blocks), then scans its own chunk.
-#define ZMAP_THREADS 256
-#define ZMAP_PER_THREAD 8
+#define ZMAP_THREADS 1024
+#define ZMAP_PER_THREAD 2
 #define ZMAP_CHUNK (ZMAP_THREADS * ZMAP_PER_THREAD)
 __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restrict__ mask, int* __restrict__ zidx,
                                                             int* __restrict__ zlist, int* __restrict__ zcount,

@@ -218,13 +218,18 @@ col_kernel(const ColArgs a) {
     using E = LineFFT<P, true, L>;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL;
     extern __shared__ float2 smem[];
+    const int tiles = (a.es + L - 1) / L;
+    const long long o = blockIdx.x / tiles;           // outer index
+    const int i_base = (int)(blockIdx.x % tiles) * L;
+    if (MODE == COL_Z) {
+        // lines are ranks of sampled positions: blocks beyond the sampled count leave at once
+        const long long bt0 = (o / ((long long)a.C * a.T)) * a.T + (o % a.T);
+        if (i_base >= a.zcount[bt0]) return;
+    }
     const typename E::Ids d = E::ids(threadIdx.x);
     typename E::Tw tw;
     E::make_tw(d, tw);
 
-    const int tiles = (a.es + L - 1) / L;
-    const long long o = blockIdx.x / tiles;           // outer index
-    const int i_base = (int)(blockIdx.x % tiles) * L;
     // COL mode: every stage sees the same line index l = tid % L
     const int i = i_base + d.l0;
     const bool line_ok = i < a.es;

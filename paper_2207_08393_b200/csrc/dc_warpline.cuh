@@ -39,7 +39,8 @@ struct WarpLine {
     static constexpr int KCAP = (MODE == ROW_INV) ? N : (((N + 3) / 4 + 1) / 2 * 2);
     static constexpr int KTILE = LW * KCAP;
     static constexpr bool HAS_K = (MODE == ROW_INV) || (MODE == ROW_FUSED && HAS_Z);
-    static constexpr bool HAS_X = (MODE != ROW_INV), HAS_M = (MODE == ROW_FUSED), HAS_I = (MODE == ROW_FUSED && HAS_Z);
+    static constexpr bool HAS_X = (MODE == ROW_FUSED);   // ROW_FWD and ROW_INV keep x in registers
+    static constexpr bool HAS_M = (MODE == ROW_FUSED), HAS_I = (MODE == ROW_FUSED && HAS_Z);
     static constexpr int OFF_S = 0, OFF_K = 2 * TILE, OFF_X = OFF_K + (HAS_K ? 2 * KTILE : 0),
                          OFF_EX = OFF_X + (HAS_X ? TILE : 0), OFF_M2 = OFF_EX + LW * EXL + (LW * EXL) % 2;
     static constexpr int OFF_IDX = OFF_M2 + (HAS_M ? TILE / 2 : 0);     // ranks of the raw k indices (ints)
@@ -144,7 +145,7 @@ warpline_kernel(const RowArgs a) {
         cp_async_commit();
 
         cf acc[R0];
-        cf xreg[R0];     // ROW_INV: x is needed only for the final update; fetched early, held in registers
+        cf xreg[R0];     // ROW_FWD / ROW_INV: x fetched once per group and held in registers
         if (!WL::HAS_X && a0 && row_ok) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) xreg[m] = a.x[x_off + j + P::BF0 * m];
@@ -167,7 +168,7 @@ warpline_kernel(const RowArgs a) {
             if (MODE != ROW_INV) {
                 if (a0) {
 #pragma unroll
-                    for (int m = 0; m < R0; ++m) v[m] = cmul(cS[j + P::BF0 * m], cX[j + P::BF0 * m]);
+                    for (int m = 0; m < R0; ++m) v[m] = cmul(cS[j + P::BF0 * m], WL::HAS_X ? cX[j + P::BF0 * m] : xreg[m]);
                     Dft<R0, -1>::run(v);
                 }
                 if (P::S == 2) {

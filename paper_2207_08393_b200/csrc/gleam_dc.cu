@@ -105,14 +105,16 @@ struct Layout {
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
-// Target size of the 3-D chunk workspace: it has to stay inside L2 between the three kernels of a
-// chunk.  GLEAM_CHUNK_MB overrides the default (tuning aid, read once).
+// Target size of the 3-D chunk workspace.  A chunk of about 48 MB would stay inside L2 between the
+// three kernels of a chunk, but at their present speed the kernels are bound by instruction issue,
+// not by bandwidth, and fewer, larger launches measure faster; the default therefore covers the
+// whole volume up to 2 GB.  GLEAM_CHUNK_MB overrides it (tuning aid, read once).
 static uint64_t chunk_target_bytes() {
     static uint64_t v = 0;
     if (v == 0) {
         const char* e = getenv("GLEAM_CHUNK_MB");
         long mb = e ? atol(e) : 0;
-        v = (uint64_t)((mb > 0 && mb <= 4096) ? mb : 48) << 20;
+        v = (uint64_t)((mb > 0 && mb <= 65536) ? mb : 2048) << 20;
     }
     return v;
 }

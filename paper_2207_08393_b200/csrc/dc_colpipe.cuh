@@ -4,8 +4,8 @@
 // A block is persistent: it walks over tiles of L neighbouring strided lines and, while it
 // transforms one tile, the next one streams from the (L2-resident) workspace into shared memory
 // with cp.async.  Three shared-memory buffers rotate between the roles "incoming tile",
-// "forward exchange" (the buffer the current tile arrived in, once every thread holds its
-// elements in registers) and "inverse exchange".
+// "forward exchange" and "inverse exchange" (the buffer the current tile arrived in, once every
+// thread holds its elements in registers).
 #pragma once
 #include "dc_warpline.cuh"
 
@@ -88,8 +88,10 @@ colpipe_mid_sep_kernel(const ColArgs a) {
 #pragma unroll
             for (int k = 0; k < RL; ++k) mw[k] = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
         }
-        __syncthreads();          // all elements are in registers: `cur` becomes the forward exchange
-        E::forward_xy(v, u, tw, d, cur, cur);
+        // forward exchange in `spare` (free since the barrier above); every thread has read its
+        // elements from `cur` before it passes the barrier inside forward_xy, so `cur` can take
+        // the inverse exchange afterwards
+        E::forward_xy(v, u, tw, d, spare, spare);
         if (actL) {
             const cf* zz = a.zin ? a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe : nullptr;
             const int* zi = a.zidx + bt * pe + i;
@@ -103,7 +105,7 @@ colpipe_mid_sep_kernel(const ColArgs a) {
                 }
             }
         }
-        E::inverse_xy(u, v, tw, d, spare, spare);
+        E::inverse_xy(u, v, tw, d, cur, cur);
         if (act0) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) a.W[base + (long long)(d.j0 + P::BF0 * m) * a.es] = v[m];

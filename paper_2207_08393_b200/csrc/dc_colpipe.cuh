@@ -17,10 +17,12 @@ struct ColPipe {
     static constexpr int BUFSZ = L * cmax(P::BUF, P::N);            // elements per buffer
     static constexpr size_t SMEM_BYTES = sizeof(cf) * (3 * BUFSZ + 2);
     static constexpr int THREADS = LineFFT<P, true, L>::THREADS;
+    // resident blocks per SM that shared memory allows (227 KB usable), capped at 3
+    static constexpr int MIN_BLOCKS = (3 * SMEM_BYTES <= 227 * 1024) ? 3 : ((2 * SMEM_BYTES <= 227 * 1024) ? 2 : 1);
 };
 
 template <class P, int L>
-__global__ void __launch_bounds__(ColPipe<P, L>::THREADS, 3)
+__global__ void __launch_bounds__(ColPipe<P, L>::THREADS, ColPipe<P, L>::MIN_BLOCKS)
 colpipe_mid_sep_kernel(const ColArgs a) {
     using E = LineFFT<P, true, L>;
     using CP = ColPipe<P, L>;

@@ -216,3 +216,32 @@ def test_chained_iterations_match_oracle(oracle):
         gg = run_gpu(gg, None, inp["sens"], inp["mask"], w.eta, 2, 0, MASK_READOUT_INVARIANT)
         go = oracle.dc_vjp(go, inp["sens"], inp["mask"], w.eta, d).astype(np.complex64)
     assert_close(gg, go, inp["g"], "chain vjp")
+
+
+def test_rank3_chunked_workspace_matches_whole_volume(oracle, tmp_path):
+    """The 3-D separable path can process the readout slabs in chunks (GLEAM_CHUNK_MB, read once per
+    process): a child process with a 1 MB chunk target must give the same bits as the default
+    whole-volume run, and both must match the oracle."""
+    import os
+    import subprocess
+    import sys
+    import paper_2207_08393_b200 as g
+    d, x, y, sens, mask = problem(3, 1, 4, 1, (12, 64, 48), MASK_READOUT_INVARIANT, seed=21, density=0.15)
+    whole = run_gpu(x, y, sens, mask, 0.9, 3, 0, MASK_READOUT_INVARIANT)
+    assert_close(whole, oracle.dc_forward(x, y, sens, mask, 0.9, d), x, "whole volume")
+    np.savez(tmp_path / "in.npz", x=x, y=y, sens=sens, mask=mask)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import sys, numpy as np; sys.path.insert(0, %r)\n"
+        "from tests.gpu_common import run_gpu\n"
+        "import paper_2207_08393_b200 as g\n"
+        "z = np.load(%r)\n"
+        "ws = g.gleam_dc_workspace_size(g.make_dims(1, 4, 1, 3, (12, 64, 48)))\n"
+        "out = run_gpu(z['x'], z['y'], z['sens'], z['mask'], 0.9, 3, 0, 1)\n"
+        "np.savez(%r, out=out, ws=ws)\n"
+    ) % (root, str(tmp_path / "in.npz"), str(tmp_path / "out.npz"))
+    # 4 coils x 64 x 48 x 8 B = 98 KB per slab: a 1 MB target gives 10 slabs per chunk, two chunks for 12 slabs
+    subprocess.run([sys.executable, "-c", code], check=True, env=dict(os.environ, GLEAM_CHUNK_MB="1"), timeout=600)
+    res = np.load(tmp_path / "out.npz")
+    assert int(res["ws"]) < g.gleam_dc_workspace_size(g.make_dims(1, 4, 1, 3, (12, 64, 48)))
+    assert np.array_equal(res["out"], whole)

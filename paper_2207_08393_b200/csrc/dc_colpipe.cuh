@@ -35,13 +35,18 @@ colpipe_mid_sep_kernel(const ColArgs a) {
 
     // tile counters are 32-bit (the launcher refuses more than 2^31 tiles): no 64-bit divisions
     const unsigned tiles_per_o = (unsigned)((a.es + L - 1) / L);
-    const unsigned ntiles = (unsigned)a.nouter * tiles_per_o;
     const long long pe = (long long)a.n1 * a.n2;
 
-    // stream tile `tile` into `dst` in [n][l] layout; chunks of 16 bytes (two neighbouring lines)
-    auto issue = [&](unsigned tile, cf* dst) {
-        const unsigned o = tile / tiles_per_o;
-        const int i_base = (int)(tile - o * tiles_per_o) * L;
+    // Work order: the grid is a whole number of "rows" of tiles_per_o blocks; block b keeps column
+    // tile b % tiles_per_o and walks over the outer indices o = b / tiles_per_o, + rows, ...  so the
+    // mask weights of its k-space entries stay in registers from one tile to the next.
+    const unsigned col_tile = blockIdx.x % tiles_per_o;
+    const unsigned rows = gridDim.x / tiles_per_o;            // host launches a multiple of tiles_per_o
+    const unsigned nout = (unsigned)a.nouter;
+
+    // stream the tile of outer index o into `dst` in [n][l] layout; chunks of 16 bytes
+    auto issue = [&](unsigned o, cf* dst) {
+        const int i_base = (int)col_tile * L;
         const cf* src = a.W + o * (long long)N * a.es + i_base;
         for (int c = threadIdx.x; c < N * (L / 2); c += CP::THREADS) {
             const int n = c / (L / 2), part = c - n * (L / 2);
@@ -49,21 +54,22 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         }
     };
 
-    unsigned tile = blockIdx.x;
-    if (tile < ntiles) issue(tile, buf[0]);
+    unsigned o = blockIdx.x / tiles_per_o;
+    if (o < nout) issue(o, buf[0]);
     cp_async_commit();
     int it = 0;
-    for (; tile < ntiles; tile += gridDim.x, ++it) {
+    long long bt_loaded = -1;
+    float mw[RL];
+    for (; o < nout; o += rows, ++it) {
         cf* cur = buf[it % 3];
         cf* nxt = buf[(it + 1) % 3];
         cf* spare = buf[(it + 2) % 3];
         cp_async_wait<0>();
         __syncthreads();          // tile is visible to all; every thread has left the previous tile
-        if (tile + gridDim.x < ntiles) issue(tile + gridDim.x, nxt);
+        if (o + rows < nout) issue(o + rows, nxt);
         cp_async_commit();
 
-        const unsigned o = tile / tiles_per_o;
-        const int i_base = (int)(tile - o * tiles_per_o) * L;
+        const int i_base = (int)col_tile * L;
         const int i = i_base + d.l0;
         const bool line_ok = i < a.es;
         const bool act0 = d.a0 && line_ok, actL = d.aL && line_ok;
@@ -77,7 +83,6 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         const long long bt = (long long)b * a.T + t;
 
         cf v[R0], u[RL];
-        float mw[RL];
         if (act0) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) v[m] = cur[(d.j0 + P::BF0 * m) * L + d.l0];
@@ -85,7 +90,8 @@ colpipe_mid_sep_kernel(const ColArgs a) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) v[m] = make_float2(0.f, 0.f);
         }
-        if (actL) {   // mask weights of this thread's k-space entries, issued early
+        if (actL && bt != bt_loaded) {   // mask weights of this thread's k-space entries: reloaded only when (b,t) changes
+            bt_loaded = bt;
             const float* mk = a.mask + bt * pe + shift_half(i, a.n2);
 #pragma unroll
             for (int k = 0; k < RL; ++k) mw[k] = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];

@@ -100,10 +100,15 @@ inline cudaError_t launch_colpipe(const ColArgs& a, cudaStream_t s) {
                                                                CP::SMEM_BYTES)) != cudaSuccess) return e;
         slots = sms * (per_sm > 0 ? per_sm : 1);
     }
-    const long long tiles = a.nouter * ((a.es + L - 1) / L);
+    const long long tiles_per_o = (a.es + L - 1) / L;
+    const long long tiles = a.nouter * tiles_per_o;
     if (tiles <= 0) return cudaSuccess;
-    if (tiles >= 2147483647LL) return cudaErrorInvalidConfiguration;
-    const long long blocks = tiles < slots ? tiles : slots;
+    if (tiles >= 2147483647LL || a.nouter >= 2147483647LL) return cudaErrorInvalidConfiguration;
+    // a whole number of rows of tiles_per_o blocks (each block keeps one column tile)
+    long long rows = slots / tiles_per_o;
+    if (rows < 1) rows = 1;
+    if (rows > a.nouter) rows = a.nouter;
+    const long long blocks = rows * tiles_per_o;
     colpipe_mid_sep_kernel<P, L><<<(unsigned)blocks, CP::THREADS, CP::SMEM_BYTES, s>>>(a);
     return cudaGetLastError();
 }

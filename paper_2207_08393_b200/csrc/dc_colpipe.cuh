@@ -21,7 +21,9 @@ struct ColPipe {
     static constexpr int MIN_BLOCKS = (3 * SMEM_BYTES <= 227 * 1024) ? 3 : ((2 * SMEM_BYTES <= 227 * 1024) ? 2 : 1);
 };
 
-template <class P, int L>
+// HAS_Z = true is the forward call: the block keeps, instead of the mask weights, the ranks of its
+// k-space entries among the sampled positions and fetches weight and z value by rank.
+template <class P, int L, bool HAS_Z>
 __global__ void __launch_bounds__(ColPipe<P, L>::THREADS, ColPipe<P, L>::MIN_BLOCKS)
 colpipe_mid_sep_kernel(const ColArgs a) {
     using E = LineFFT<P, true, L>;
@@ -59,7 +61,8 @@ colpipe_mid_sep_kernel(const ColArgs a) {
     cp_async_commit();
     int it = 0;
     long long bt_loaded = -1;
-    float mw[RL];
+    float mw[RL];       // VJP: mask weights of this thread's k-space entries
+    int zr[RL];         // forward: their ranks among the sampled positions (-1: unsampled)
     for (; o < nout; o += rows, ++it) {
         cf* cur = buf[it % 3];
         cf* nxt = buf[(it + 1) % 3];
@@ -92,25 +95,37 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         }
         if (actL && bt != bt_loaded) {   // mask weights of this thread's k-space entries: reloaded only when (b,t) changes
             bt_loaded = bt;
-            const float* mk = a.mask + bt * pe + shift_half(i, a.n2);
+            if (HAS_Z) {
+                const int* zi = a.zidx + bt * pe + i;
 #pragma unroll
-            for (int k = 0; k < RL; ++k) mw[k] = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
+                for (int k = 0; k < RL; ++k) zr[k] = zi[(long long)(d.jL + P::BFL * k) * a.n2];
+            } else {
+                const float* mk = a.mask + bt * pe + shift_half(i, a.n2);
+#pragma unroll
+                for (int k = 0; k < RL; ++k) mw[k] = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
+            }
         }
         // forward exchange in `spare` (free since the barrier above); every thread has read its
         // elements from `cur` before it passes the barrier inside forward_xy, so `cur` can take
         // the inverse exchange afterwards
         E::forward_xy(v, u, tw, d, spare, spare);
         if (actL) {
-            const cf* zz = a.zin ? a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe : nullptr;
-            const int* zi = a.zidx + bt * pe + i;
+            if (HAS_Z) {
+                const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
+                const float* m2 = a.m2c + bt * pe;
 #pragma unroll
-            for (int k = 0; k < RL; ++k) {
-                const float w = mw[k] * mw[k] * a.scale2;
-                u[k] = cscale(u[k], w);
-                if (zz && mw[k] != 0.f) {
-                    const cf q = zz[zi[(long long)(d.jL + P::BFL * k) * a.n2]];
-                    u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
+                for (int k = 0; k < RL; ++k) {
+                    if (zr[k] >= 0) {
+                        const float w = m2[zr[k]] * a.scale2;
+                        const cf q = zz[zr[k]];
+                        u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
+                    } else {
+                        u[k] = make_float2(0.f, 0.f);
+                    }
                 }
+            } else {
+#pragma unroll
+                for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], mw[k] * mw[k] * a.scale2);
             }
         }
         E::inverse_xy(u, v, tw, d, cur, cur);

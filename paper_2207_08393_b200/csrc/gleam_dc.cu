@@ -44,7 +44,7 @@ static const SizeOps* find_size(int n) {
 #define ZMAP_CHUNK (ZMAP_THREADS * ZMAP_PER_THREAD)
 __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restrict__ mask, int* __restrict__ zidx,
                                                             int* __restrict__ zlist, int* __restrict__ zcount,
-                                                            int n1, int n2, int rank) {
+                                                            float* __restrict__ m2c, int n1, int n2, int rank) {
     __shared__ int warp_sum[ZMAP_THREADS / 32];
     __shared__ int base_sh;
     const int pe = (rank == 2) ? n2 : n1 * n2;
@@ -87,7 +87,10 @@ __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restr
     for (int e = 0; e < ZMAP_PER_THREAD; ++e) {
         const int q = q0 + e;
         if (q >= pe) break;
-        if (on[e]) { zidx[bt * pe + q] = r; zlist[bt * pe + r] = src[e]; ++r; }
+        if (on[e]) {
+            const float mv = mk[src[e]];
+            zidx[bt * pe + q] = r; zlist[bt * pe + r] = src[e]; m2c[bt * pe + r] = mv * mv; ++r;
+        }
         else zidx[bt * pe + q] = -1;
     }
     if (q_begin + ZMAP_CHUNK >= pe && tid == ZMAP_THREADS - 1) zcount[bt] = r;   // last chunk, last thread: total
@@ -101,7 +104,7 @@ struct Layout {
     long long V, units, images;
     bool separable;
     // workspace (byte offsets)
-    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_W, total;
+    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_m2c, off_W, total;
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
@@ -139,7 +142,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     if (L->images * L->n0 * L->n1 >= (1ll << 31)) return GLEAM_ERR_BAD_DIMS;   // row counters are 32-bit
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
-    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_W = 0; L->G = 0;
+    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_m2c = L->off_W = 0; L->G = 0;
     if (L->separable) {
         const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
         if (with_y) {
@@ -148,6 +151,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
             L->off_zidx = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(int), 256);
             L->off_zlist = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(int), 256);
             L->off_zcount = off; off = align_up(off + (uint64_t)L->images * sizeof(int), 256);
+            L->off_m2c = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(float), 256);
         }
         if (L->rank == 3) {
             const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
@@ -267,11 +271,12 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             int* zidx = (int*)(ws + L.off_zidx);
             int* zlist = (int*)(ws + L.off_zlist);
             int* zcount = (int*)(ws + L.off_zcount);
+            float* m2c = (float*)(ws + L.off_m2c);
             CK(prof_mark(GLEAM_K_PREP_M2, s));
             zmap_kernel<<<dim3((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images), ZMAP_THREADS, 0, s>>>(
-                mask, zidx, zlist, zcount, L.n1, L.n2, L.rank);
+                mask, zidx, zlist, zcount, m2c, L.n1, L.n2, L.rank);
             CK(cudaGetLastError());
-            ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount;
+            ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount; ca.m2c = m2c;
             ra.zidx = zidx;
             ColArgs cz = ca;
             cz.y = (const cf*)y; cz.z = z; cz.mask = mask;

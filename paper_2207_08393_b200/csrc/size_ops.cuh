@@ -85,18 +85,18 @@ inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
 }
 
 // persistent launch of the pipelined column kernel (separable 3-D path)
-template <class P, int L>
-inline cudaError_t launch_colpipe(const ColArgs& a, cudaStream_t s) {
+template <class P, int L, bool HAS_Z>
+inline cudaError_t launch_colpipe_z(const ColArgs& a, cudaStream_t s) {
     using CP = ColPipe<P, L>;
     static bool attr_done = false;
     static int slots = 0;
-    cudaError_t e = ensure_smem(colpipe_mid_sep_kernel<P, L>, CP::SMEM_BYTES, attr_done);
+    cudaError_t e = ensure_smem(colpipe_mid_sep_kernel<P, L, HAS_Z>, CP::SMEM_BYTES, attr_done);
     if (e != cudaSuccess) return e;
     if (slots == 0) {
         int dev = 0, sms = 0, per_sm = 0;
         if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, colpipe_mid_sep_kernel<P, L>, CP::THREADS,
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, colpipe_mid_sep_kernel<P, L, HAS_Z>, CP::THREADS,
                                                                CP::SMEM_BYTES)) != cudaSuccess) return e;
         slots = sms * (per_sm > 0 ? per_sm : 1);
     }
@@ -109,8 +109,13 @@ inline cudaError_t launch_colpipe(const ColArgs& a, cudaStream_t s) {
     if (rows < 1) rows = 1;
     if (rows > a.nouter) rows = a.nouter;
     const long long blocks = rows * tiles_per_o;
-    colpipe_mid_sep_kernel<P, L><<<(unsigned)blocks, CP::THREADS, CP::SMEM_BYTES, s>>>(a);
+    colpipe_mid_sep_kernel<P, L, HAS_Z><<<(unsigned)blocks, CP::THREADS, CP::SMEM_BYTES, s>>>(a);
     return cudaGetLastError();
+}
+
+template <class P, int L>
+inline cudaError_t launch_colpipe(const ColArgs& a, cudaStream_t s) {
+    return a.zin ? launch_colpipe_z<P, L, true>(a, s) : launch_colpipe_z<P, L, false>(a, s);
 }
 
 template <class P, int LR, class PC, int LC>

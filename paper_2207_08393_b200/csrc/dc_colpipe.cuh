@@ -113,14 +113,28 @@ colpipe_mid_sep_kernel(const ColArgs a) {
             if (HAS_Z) {
                 const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
                 const float* m2 = a.m2c + bt * pe;
+                // branch-free gathers in batches of ZB entries (unsampled entries read rank 0 and
+                // discard it), so that the loads of a batch are in flight together
+                constexpr int ZB = 5;
 #pragma unroll
-                for (int k = 0; k < RL; ++k) {
-                    if (zr[k] >= 0) {
-                        const float w = m2[zr[k]] * a.scale2;
-                        const cf q = zz[zr[k]];
-                        u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
-                    } else {
-                        u[k] = make_float2(0.f, 0.f);
+                for (int k0 = 0; k0 < RL; k0 += ZB) {
+                    cf q[ZB]; float w[ZB];
+#pragma unroll
+                    for (int e = 0; e < ZB; ++e) {
+                        if (k0 + e < RL) {
+                            const int r = zr[k0 + e] >= 0 ? zr[k0 + e] : 0;
+                            q[e] = zz[r];
+                            w[e] = m2[r];
+                        }
+                    }
+#pragma unroll
+                    for (int e = 0; e < ZB; ++e) {
+                        if (k0 + e < RL) {
+                            const int k = k0 + e;
+                            const float ws = (zr[k] >= 0) ? w[e] * a.scale2 : 0.f;
+                            const float zs = (zr[k] >= 0) ? 1.f : 0.f;
+                            u[k] = make_float2(fmaf(ws, u[k].x, -zs * q[e].x), fmaf(ws, u[k].y, -zs * q[e].y));
+                        }
                     }
                 }
             } else {

@@ -42,6 +42,7 @@ static const SizeOps* find_size(int n) {
 #define ZMAP_THREADS 1024
 #define ZMAP_PER_THREAD 2
 #define ZMAP_CHUNK (ZMAP_THREADS * ZMAP_PER_THREAD)
+#define ZMAP_TILE 8
 __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restrict__ mask, int* __restrict__ zidx,
                                                             int* __restrict__ zlist, int* __restrict__ zcount,
                                                             float* __restrict__ m2c, int n1, int n2, int rank) {
@@ -52,9 +53,20 @@ __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restr
     const float* mk = mask + bt * pe;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q_begin = blockIdx.x * ZMAP_CHUNK;
-    auto src_of = [&](int q) -> int {
-        if (rank == 2) return shift_half(q, n2);
-        return shift_half(q / n2, n1) * n2 + shift_half(q % n2, n2);
+    // Rank order.  rank 2: the raw k index.  rank 3: column tiles of ZMAP_TILE raw kz indices, inside
+    // a tile by (raw ky, raw kz): the sampled entries that one tile of the column kernel needs are
+    // then neighbours in the compact z table.  raw_of maps the scan position to the raw position.
+    const bool tiled = (rank == 3) && (n2 % ZMAP_TILE == 0);
+    auto raw_of = [&](int q) -> int {
+        if (!tiled) return q;
+        const int per_tile = n1 * ZMAP_TILE;
+        const int tile = q / per_tile, rem = q - tile * per_tile;
+        return (rem / ZMAP_TILE) * n2 + tile * ZMAP_TILE + rem % ZMAP_TILE;
+    };
+    auto src_of = [&](int q) -> int {            // unshifted source position of scan position q
+        const int rq = raw_of(q);
+        if (rank == 2) return shift_half(rq, n2);
+        return shift_half(rq / n2, n1) * n2 + shift_half(rq % n2, n2);
     };
     // sampled positions before this chunk
     int c = 0;
@@ -89,9 +101,9 @@ __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restr
         if (q >= pe) break;
         if (on[e]) {
             const float mv = mk[src[e]];
-            zidx[bt * pe + q] = r; zlist[bt * pe + r] = src[e]; m2c[bt * pe + r] = mv * mv; ++r;
+            zidx[bt * pe + raw_of(q)] = r; zlist[bt * pe + r] = src[e]; m2c[bt * pe + r] = mv * mv; ++r;
         }
-        else zidx[bt * pe + q] = -1;
+        else zidx[bt * pe + raw_of(q)] = -1;
     }
     if (q_begin + ZMAP_CHUNK >= pe && tid == ZMAP_THREADS - 1) zcount[bt] = r;   // last chunk, last thread: total
 }

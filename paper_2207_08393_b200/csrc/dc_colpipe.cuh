@@ -11,12 +11,18 @@
 
 namespace gleam {
 
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(d), "l"(gsrc) : "memory");
+}
+
 template <class P, int L>
 struct ColPipe {
     static constexpr bool ELIGIBLE = (P::S == 2) && (L % 2 == 0);
     static constexpr int BUFSZ = L * cmax(P::BUF, P::N);            // elements per buffer
     static constexpr size_t SMEM_BYTES = sizeof(cf) * (3 * BUFSZ + 2);
     static constexpr int THREADS = LineFFT<P, true, L>::THREADS;
+    static constexpr int ZCAP = 384;      // sampled entries per tile whose z values are staged (forward call)
     // resident blocks per SM that shared memory allows (227 KB usable), capped at 3
     static constexpr int MIN_BLOCKS = (3 * SMEM_BYTES <= 227 * 1024) ? 3 : ((2 * SMEM_BYTES <= 227 * 1024) ? 2 : 1);
 };
@@ -47,6 +53,22 @@ colpipe_mid_sep_kernel(const ColArgs a) {
     const unsigned nout = (unsigned)a.nouter;
 
     // stream the tile of outer index o into `dst` in [n][l] layout; chunks of 16 bytes
+    __shared__ int s_rank[HAS_Z ? CP::ZCAP : 1];        // ranks of the tile's sampled entries (forward call)
+    __shared__ float s_wt[HAS_Z ? CP::ZCAP : 1];        // their scaled squared mask weights
+    __shared__ cf s_z[2][HAS_Z ? CP::ZCAP : 1];         // their z values, double-buffered over tiles
+    __shared__ int s_wcnt[CP::THREADS / 32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int z_total = 0;            // sampled entries of this block's column tile
+    bool z_staged = false;      // they fit the staging area
+
+    // z values of the tile of outer index o -> s_z[slot] (asynchronous, 8 bytes each)
+    auto issue_z = [&](unsigned o, int slot) {
+        const unsigned unit = o / (unsigned)a.G;
+        const int gi = (int)(o - unit * (unsigned)a.G);
+        const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
+        for (int e = threadIdx.x; e < z_total; e += CP::THREADS) cp_async8(&s_z[slot][e], zz + s_rank[e]);
+    };
+
     auto issue = [&](unsigned o, cf* dst) {
         const int i_base = (int)col_tile * L;
         const cf* src = a.W + o * (long long)N * a.es + i_base;
@@ -93,54 +115,78 @@ colpipe_mid_sep_kernel(const ColArgs a) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) v[m] = make_float2(0.f, 0.f);
         }
-        if (actL && bt != bt_loaded) {   // mask weights of this thread's k-space entries: reloaded only when (b,t) changes
+        if (bt != bt_loaded) {   // per-(b,t) tables of this thread's k-space entries: reloaded only when (b,t) changes
             bt_loaded = bt;
             if (HAS_Z) {
+                // Ranks of this thread's entries among the sampled positions.  The sampled entries of
+                // the whole tile are then numbered block-wide; their ranks and weights go to shared
+                // memory, and every later tile fetches its z values asynchronously, one tile ahead.
                 const int* zi = a.zidx + bt * pe + i;
+                const float* m2 = a.m2c + bt * pe;
 #pragma unroll
-                for (int k = 0; k < RL; ++k) zr[k] = zi[(long long)(d.jL + P::BFL * k) * a.n2];
-            } else {
+                for (int k = 0; k < RL; ++k) zr[k] = actL ? zi[(long long)(d.jL + P::BFL * k) * a.n2] : -1;
+                int wc = 0;
+#pragma unroll
+                for (int k = 0; k < RL; ++k) wc += __popc(__ballot_sync(0xffffffffu, zr[k] >= 0));
+                __syncthreads();                       // earlier readers of the tables are done
+                if (lane == 0) s_wcnt[warp] = wc;
+                __syncthreads();
+                int base = 0, total = 0;
+                for (int w2 = 0; w2 < CP::THREADS / 32; ++w2) { if (w2 < warp) base += s_wcnt[w2]; total += s_wcnt[w2]; }
+                z_total = total;
+                z_staged = total <= CP::ZCAP;
+                if (z_staged) {
+#pragma unroll
+                    for (int k = 0; k < RL; ++k) {
+                        const bool on = zr[k] >= 0;
+                        const unsigned bal = __ballot_sync(0xffffffffu, on);
+                        if (on) {
+                            const int pos = base + __popc(bal & ((1u << lane) - 1u));
+                            s_rank[pos] = zr[k];
+                            s_wt[pos] = m2[zr[k]] * a.scale2;
+                            zr[k] = pos;
+                        }
+                        base += __popc(bal);
+                    }
+                    __syncthreads();
+                    issue_z(o, it & 1);                // this tile's values were not prefetched
+                    cp_async_commit();
+                    cp_async_wait<0>();
+                    __syncthreads();
+                }
+            } else if (actL) {
                 const float* mk = a.mask + bt * pe + shift_half(i, a.n2);
 #pragma unroll
                 for (int k = 0; k < RL; ++k) mw[k] = mk[(long long)shift_half(d.jL + P::BFL * k, N) * a.n2];
             }
         }
+        if (HAS_Z && z_staged && o + rows < nout) {   // z values of the next tile, one tile ahead
+            issue_z(o + rows, (it + 1) & 1);
+            cp_async_commit();
+        }
         // forward exchange in `spare` (free since the barrier above); every thread has read its
         // elements from `cur` before it passes the barrier inside forward_xy, so `cur` can take
         // the inverse exchange afterwards
         E::forward_xy(v, u, tw, d, spare, spare);
-        if (actL) {
-            if (HAS_Z) {
+        if (HAS_Z) {
+            if (actL) {
                 const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
                 const float* m2 = a.m2c + bt * pe;
-                // branch-free gathers in batches of ZB entries (unsampled entries read rank 0 and
-                // discard it), so that the loads of a batch are in flight together
-                constexpr int ZB = 5;
+                const cf* zs = s_z[it & 1];
 #pragma unroll
-                for (int k0 = 0; k0 < RL; k0 += ZB) {
-                    cf q[ZB]; float w[ZB];
-#pragma unroll
-                    for (int e = 0; e < ZB; ++e) {
-                        if (k0 + e < RL) {
-                            const int r = zr[k0 + e] >= 0 ? zr[k0 + e] : 0;
-                            q[e] = zz[r];
-                            w[e] = m2[r];
-                        }
-                    }
-#pragma unroll
-                    for (int e = 0; e < ZB; ++e) {
-                        if (k0 + e < RL) {
-                            const int k = k0 + e;
-                            const float ws = (zr[k] >= 0) ? w[e] * a.scale2 : 0.f;
-                            const float zs = (zr[k] >= 0) ? 1.f : 0.f;
-                            u[k] = make_float2(fmaf(ws, u[k].x, -zs * q[e].x), fmaf(ws, u[k].y, -zs * q[e].y));
-                        }
+                for (int k = 0; k < RL; ++k) {
+                    if (zr[k] >= 0) {
+                        const float w = z_staged ? s_wt[zr[k]] : m2[zr[k]] * a.scale2;
+                        const cf q = z_staged ? zs[zr[k]] : zz[zr[k]];
+                        u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
+                    } else {
+                        u[k] = make_float2(0.f, 0.f);
                     }
                 }
-            } else {
-#pragma unroll
-                for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], mw[k] * mw[k] * a.scale2);
             }
+        } else if (actL) {
+#pragma unroll
+            for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], mw[k] * mw[k] * a.scale2);
         }
         E::inverse_xy(u, v, tw, d, cur, cur);
         if (act0) {

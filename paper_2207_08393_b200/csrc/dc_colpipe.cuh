@@ -53,9 +53,11 @@ colpipe_mid_sep_kernel(const ColArgs a) {
     const unsigned nout = (unsigned)a.nouter;
 
     // stream the tile of outer index o into `dst` in [n][l] layout; chunks of 16 bytes
+    // slot ZCAP of s_wt / s_z is a dummy that holds zero: unsampled entries point at it, which keeps
+    // the k-space update free of branches
     __shared__ int s_rank[HAS_Z ? CP::ZCAP : 1];        // ranks of the tile's sampled entries (forward call)
-    __shared__ float s_wt[HAS_Z ? CP::ZCAP : 1];        // their scaled squared mask weights
-    __shared__ cf s_z[2][HAS_Z ? CP::ZCAP : 1];         // their z values, double-buffered over tiles
+    __shared__ float s_wt[HAS_Z ? CP::ZCAP + 1 : 1];    // their scaled squared mask weights
+    __shared__ cf s_z[2][HAS_Z ? CP::ZCAP + 1 : 1];     // their z values, double-buffered over tiles
     __shared__ int s_wcnt[CP::THREADS / 32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int z_total = 0;            // sampled entries of this block's column tile
@@ -136,6 +138,11 @@ colpipe_mid_sep_kernel(const ColArgs a) {
                 z_total = total;
                 z_staged = total <= CP::ZCAP;
                 if (z_staged) {
+                    if (threadIdx.x == 0) {
+                        s_wt[CP::ZCAP] = 0.f;
+                        s_z[0][CP::ZCAP] = make_float2(0.f, 0.f);
+                        s_z[1][CP::ZCAP] = make_float2(0.f, 0.f);
+                    }
 #pragma unroll
                     for (int k = 0; k < RL; ++k) {
                         const bool on = zr[k] >= 0;
@@ -145,6 +152,8 @@ colpipe_mid_sep_kernel(const ColArgs a) {
                             s_rank[pos] = zr[k];
                             s_wt[pos] = m2[zr[k]] * a.scale2;
                             zr[k] = pos;
+                        } else {
+                            zr[k] = CP::ZCAP;
                         }
                         base += __popc(bal);
                     }
@@ -169,15 +178,22 @@ colpipe_mid_sep_kernel(const ColArgs a) {
         // the inverse exchange afterwards
         E::forward_xy(v, u, tw, d, spare, spare);
         if (HAS_Z) {
-            if (actL) {
-                const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
-                const float* m2 = a.m2c + bt * pe;
+            if (actL && z_staged) {
                 const cf* zs = s_z[it & 1];
 #pragma unroll
                 for (int k = 0; k < RL; ++k) {
+                    const float w = s_wt[zr[k]];
+                    const cf q = zs[zr[k]];
+                    u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
+                }
+            } else if (actL) {     // more sampled entries than the staging area holds: fetch directly
+                const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
+                const float* m2 = a.m2c + bt * pe;
+#pragma unroll
+                for (int k = 0; k < RL; ++k) {
                     if (zr[k] >= 0) {
-                        const float w = z_staged ? s_wt[zr[k]] : m2[zr[k]] * a.scale2;
-                        const cf q = z_staged ? zs[zr[k]] : zz[zr[k]];
+                        const float w = m2[zr[k]] * a.scale2;
+                        const cf q = zz[zr[k]];
                         u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
                     } else {
                         u[k] = make_float2(0.f, 0.f);

@@ -86,7 +86,8 @@ colpipe_mid_sep_kernel(const ColArgs a) {
     int it = 0;
     long long bt_loaded = -1;
     float mw[RL];       // VJP: mask weights of this thread's k-space entries
-    int zr[RL];         // forward: their ranks among the sampled positions (-1: unsampled)
+    unsigned zp[(RL + 1) / 2];   // forward: positions of this thread's entries in the tile's staged list, two
+                                 // 16-bit values per register (ZCAP = the zero dummy slot: unsampled entry)
     for (; o < nout; o += rows, ++it) {
         cf* cur = buf[it % 3];
         cf* nxt = buf[(it + 1) % 3];
@@ -125,6 +126,7 @@ colpipe_mid_sep_kernel(const ColArgs a) {
                 // memory, and every later tile fetches its z values asynchronously, one tile ahead.
                 const int* zi = a.zidx + bt * pe + i;
                 const float* m2 = a.m2c + bt * pe;
+                int zr[RL];
 #pragma unroll
                 for (int k = 0; k < RL; ++k) zr[k] = actL ? zi[(long long)(d.jL + P::BFL * k) * a.n2] : -1;
                 int wc = 0;
@@ -147,14 +149,14 @@ colpipe_mid_sep_kernel(const ColArgs a) {
                     for (int k = 0; k < RL; ++k) {
                         const bool on = zr[k] >= 0;
                         const unsigned bal = __ballot_sync(0xffffffffu, on);
+                        int pos = CP::ZCAP;
                         if (on) {
-                            const int pos = base + __popc(bal & ((1u << lane) - 1u));
+                            pos = base + __popc(bal & ((1u << lane) - 1u));
                             s_rank[pos] = zr[k];
                             s_wt[pos] = m2[zr[k]] * a.scale2;
-                            zr[k] = pos;
-                        } else {
-                            zr[k] = CP::ZCAP;
                         }
+                        if (k % 2 == 0) zp[k / 2] = (unsigned)pos;
+                        else zp[k / 2] |= (unsigned)pos << 16;
                         base += __popc(bal);
                     }
                     __syncthreads();
@@ -182,18 +184,21 @@ colpipe_mid_sep_kernel(const ColArgs a) {
                 const cf* zs = s_z[it & 1];
 #pragma unroll
                 for (int k = 0; k < RL; ++k) {
-                    const float w = s_wt[zr[k]];
-                    const cf q = zs[zr[k]];
+                    const int pos = (k % 2 == 0) ? (int)(zp[k / 2] & 0xffffu) : (int)(zp[k / 2] >> 16);
+                    const float w = s_wt[pos];
+                    const cf q = zs[pos];
                     u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
                 }
             } else if (actL) {     // more sampled entries than the staging area holds: fetch directly
                 const cf* zz = a.zin + ((long long)unit * a.n0 + a.i0_start + gi) * pe;
                 const float* m2 = a.m2c + bt * pe;
+                const int* zi = a.zidx + bt * pe + i;
 #pragma unroll
                 for (int k = 0; k < RL; ++k) {
-                    if (zr[k] >= 0) {
-                        const float w = m2[zr[k]] * a.scale2;
-                        const cf q = zz[zr[k]];
+                    const int r = zi[(long long)(d.jL + P::BFL * k) * a.n2];
+                    if (r >= 0) {
+                        const float w = m2[r] * a.scale2;
+                        const cf q = zz[r];
                         u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
                     } else {
                         u[k] = make_float2(0.f, 0.f);

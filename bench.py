@@ -49,7 +49,7 @@ def fp32_peak_tflops(sm_mhz):
 # ------------------------------------------------------------------------------------------------
 # roofline bookkeeping (algorithmic bytes / flops; N log2 N counting of the transforms)
 # ------------------------------------------------------------------------------------------------
-def north_star_roofline(w, with_y):
+def call_roofline(w, with_y):
     """min bytes = x + S + (y) + mask + out;  flops = 2 B C T transforms x 5 N log2 N, N = points
     per full transform."""
     img = w.batch * w.frames * w.V * 8
@@ -65,7 +65,7 @@ def north_star_roofline(w, with_y):
 
 def kernel_work(cls, w, launches_per_call):
     """Algorithmic (bytes, flops) of ONE launch of a kernel class for workload w.
-    Per voxel*coil: see the per-kernel table in the design doc."""
+    Per voxel*coil figures are listed beside each case."""
     W = w.voxel_coils / launches_per_call        # voxel*coils one launch processes
     C = w.coils
     l2 = math.log2
@@ -372,12 +372,12 @@ def run_ours(args, w):
                  "share_of_step": kd["ms_per_step"] / sum(k["ms_per_step"] for k in kernels.values())})
     ns = {}
     for name, with_y, ms in (("forward", True, split[0]), ("vjp", False, split[1])):
-        nbytes, flops = north_star_roofline(w, with_y)
+        nbytes, flops = call_roofline(w, with_y)
         t_b, t_f = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (alu_peak * 1e12)
         ns[name] = {"min_bytes": nbytes, "fft_flops": flops, "hbm_us": t_b * 1e6, "fp32_us": t_f * 1e6,
                     "measured_us": ms * 1e3, "frac": max(t_b, t_f) / (ms * 1e-3)}
 
-    # ---- CPU baseline: the oracle, once, on the GPU machine's host cores ---------------------------
+    # ---- CPU baseline: the oracle, once, on the host cores of the machine ---------------------------
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         from oracle import oracle
@@ -408,7 +408,7 @@ def run_ours(args, w):
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": int(launches),
         "roofline": roof,
-        "north_star_roofline": ns,
+        "call_roofline": ns,
         "kernels": kernels,
         "cpu_baseline": cpu,
     }

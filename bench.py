@@ -2,10 +2,12 @@
 
     python bench.py --gpus N --steps K --warmup W [--workload knee3d] [--impl reference]
 
-One step = one gleam_dc_forward followed by one gleam_dc_vjp on the same synthetic workload
-(all rows of the hot path: sensitivity multiply, FFT, mask + residual, inverse FFT, coil sum,
-update, and the VJP).  `value` is voxel*coils per second with every input resident in HBM;
-`e2e` is the same metric through the host-buffer C-ABI calls with pinned host inputs, the
+One step = the workload's unrolled iterations: `chain` gleam_dc_forward calls chained as
+x_{i+1} = DC(x_i), then `chain` gleam_dc_vjp calls chained backwards, all on the same y, S and mask
+(chain = 1 for knee3d, knee2d and slice64; 10 for brain2d; 8 for cine).  Every call runs all rows
+of the hot path: sensitivity multiply, FFT, mask + residual, inverse FFT, coil sum, update.
+`value` is voxel*coils per second with every input resident in HBM; `e2e` is the same metric
+through the host-buffer C-ABI calls (one forward + one VJP per step) with pinned host inputs, the
 host->device copies and the device->host copy of the results inside the timed region.
 
 N > 1 runs N independent replicas (the path has no exchange step); the time is the max over ranks.
@@ -248,9 +250,30 @@ def run_ours(args, w):
     gin = torch.empty_like(tg)
     stream = torch.cuda.current_stream()
 
+    chain = max(1, w.chain)
+    out2 = torch.empty_like(tx) if chain > 1 else None
+    gin2 = torch.empty_like(tg) if chain > 1 else None
+
+    def forward_chain():
+        """x_{i+1} = DC(x_i): `chain` unrolled iterations with the same y, S and mask (the learned
+        prior between them is outside this library)."""
+        src = tx
+        for i in range(chain):
+            dst = out if i % 2 == 0 else out2
+            dc.forward(src, ty, ts, tm, w.eta, dst)
+            src = dst
+
+    def vjp_chain():
+        """g_i = VJP(g_{i+1}) through the same `chain` iterations."""
+        src = tg
+        for i in range(chain):
+            dst = gin if i % 2 == 0 else gin2
+            dc.vjp(src, ts, tm, w.eta, dst)
+            src = dst
+
     def step():
-        dc.forward(tx, ty, ts, tm, w.eta, out)
-        dc.vjp(tg, ts, tm, w.eta, gin)
+        forward_chain()
+        vjp_chain()
 
     flush = None
     inputs_bytes = sum(t.numel() * t.element_size() for t in (tx, tg, ts, tm, ty))
@@ -293,7 +316,7 @@ def run_ours(args, w):
         local_ms = sum(a.elapsed_time(b) for a, b in evs)
     launches = g.gleam_dc_launch_count() - launches0
     t_end = time.time()
-    total_ms, total_units = aggregate(local_ms, w.voxel_coils * args.steps, world, dist, dev)
+    total_ms, total_units = aggregate(local_ms, w.voxel_coils * chain * args.steps, world, dist, dev)
     value = total_units / (total_ms * 1e-3)
 
     # ---- per-kernel pass (CUDA events around every launch, on the launching stream) ----------
@@ -306,7 +329,7 @@ def run_ours(args, w):
     prof = g.gleam_dc_profile_end()
     kernels = {}
     for cls, (ms, cnt) in prof.items():
-        per_call = cnt / (2.0 * prof_steps)        # launches per call, averaged over forward and vjp
+        per_call = cnt / (2.0 * chain * prof_steps)        # launches per call, averaged over forward and vjp
         nbytes, flops = kernel_work(cls, w, max(per_call, 1e-9))
         avg_s = ms * 1e-3 / cnt
         kernels[cls] = {"launches_per_step": cnt / prof_steps, "ms_per_step": ms / prof_steps, "avg_us": avg_s * 1e6,
@@ -317,11 +340,11 @@ def run_ours(args, w):
     for _ in range(prof_steps):
         if flush is not None:
             flush.fill_(1)
-        ef[0].record(stream); dc.forward(tx, ty, ts, tm, w.eta, out)
-        ef[1].record(stream); dc.vjp(tg, ts, tm, w.eta, gin)
+        ef[0].record(stream); forward_chain()
+        ef[1].record(stream); vjp_chain()
         ef[2].record(stream); torch.cuda.synchronize()
-        split[0] += ef[0].elapsed_time(ef[1]) / prof_steps
-        split[1] += ef[1].elapsed_time(ef[2]) / prof_steps
+        split[0] += ef[0].elapsed_time(ef[1]) / prof_steps / chain      # per call
+        split[1] += ef[1].elapsed_time(ef[2]) / prof_steps / chain
 
     clocks = sampler.stop(t_begin, t_end) if sampler else None
 
@@ -336,6 +359,8 @@ def run_ours(args, w):
         g.gleam_dc_forward_host(hx, hy, hs, hm, w.eta, hout, d_host, arena)
         g.gleam_dc_vjp_host(hg, hs, hm, w.eta, hgin, d_host, arena)
 
+    dc.forward(tx, ty, ts, tm, w.eta, out)      # single calls on the device-resident inputs: the
+    dc.vjp(tg, ts, tm, w.eta, gin)              # results the host-buffer path has to reproduce
     step_host()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -400,9 +425,10 @@ def run_ours(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "description": w.description, "step": "1 gleam_dc_forward + 1 gleam_dc_vjp",
-                   "voxel_coils_per_step": w.voxel_coils, "parallelism": "replicas only" if world > 1 else "1 gpu",
-                   "l2": "inputs exceed L2" if flush is None else "256 MB L2 flush before every step"},
+        "config": {"workload": w.name, "description": w.description, "step": "%d chained gleam_dc_forward + %d chained gleam_dc_vjp" % (chain, chain),
+                   "voxel_coils_per_step": w.voxel_coils * chain, "e2e_step": "1 forward + 1 vjp with host buffers", "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "inputs exceed L2" if flush is None else "256 MB L2 flush before every step (chain)"},
+        "ms_per_iteration": total_ms / args.steps / chain,
         "clocks": clocks,
         "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},

@@ -50,6 +50,7 @@ struct ColArgs {
     int C, T;
     int rank, n0, n1, n2;
     int G, i0_start;    // COL_MID_SEP chunk: slabs in the chunk, first slab
+    int ztiles;         // COL_Z: blocks launched per outer index (they stride over the tiles of ranks)
     float scale;        // COL_Z: g_ro g_pe / sqrt(N_ro N_pe);  COL_MID_FULL: g / sqrt(Ntot)
     float scale2;       // COL_MID_FULL: 1 / Ntot;  COL_MID_SEP: 1 / (n1 n2)
 };
@@ -219,9 +220,11 @@ col_kernel(const ColArgs a) {
     using E = LineFFT<P, true, L>;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL;
     extern __shared__ float2 smem[];
-    const int tiles = (a.es + L - 1) / L;
+    // COL_Z launches ztiles blocks per outer index and lets them stride over the tiles of sampled
+    // ranks (their number is only known on the device); the other modes launch one block per tile
+    const int tiles = (MODE == COL_Z) ? a.ztiles : (a.es + L - 1) / L;
     const long long o = blockIdx.x / tiles;           // outer index
-    const int i_base = (int)(blockIdx.x % tiles) * L;
+    int i_base = (int)(blockIdx.x % tiles) * L;
     if (MODE == COL_Z) {
         // lines are ranks of sampled positions: blocks beyond the sampled count leave at once
         const long long bt0 = (o / ((long long)a.C * a.T)) * a.T + (o % a.T);
@@ -232,7 +235,7 @@ col_kernel(const ColArgs a) {
     E::make_tw(d, tw);
 
     // COL mode: every stage sees the same line index l = tid % L
-    const int i = i_base + d.l0;
+    int i = i_base + d.l0;
     const bool line_ok = i < a.es;
     const bool act0 = d.a0 && line_ok, actL = d.aL && line_ok;
     const long long base = o * (long long)N * a.es + i;
@@ -240,6 +243,7 @@ col_kernel(const ColArgs a) {
     cf v[R0], u[RL];
 
     if (MODE == COL_Z) {
+      for (;; i_base += tiles * L, i += tiles * L) {
         // Lines are the sampled phase-encode positions of this unit's (b,t), by rank r.
         // z[r] = (g/sqrt(N_ro N_pe)) (-1)^{n_ro} (-1)^{p} M[p] * Rraw^H( (-1)^{k_ro} y[.., p] ),  p = zlist[r]
         const int t = (int)(o % a.T);
@@ -247,7 +251,7 @@ col_kernel(const ColArgs a) {
         const long long bt = (long long)b * a.T + t;
         const long long pe = a.es;
         const int cnt = a.zcount[bt];
-        if (i_base >= cnt) return;                      // whole block beyond the sampled set
+        if (i_base >= cnt) return;                      // no tile of sampled ranks left for this block
         const bool ok = i < cnt;
         int p = 0, psign = 0; float mv = 0.f;
         if (ok) {
@@ -273,7 +277,8 @@ col_kernel(const ColArgs a) {
                 a.z[o * (long long)N * pe + (long long)n * pe + i] = cscale(v[m], ff);
             }
         }
-        return;
+        __syncthreads();                                // exchange buffer is reused by the next tile
+      }
     }
 
     if (MODE == COL_INV) {

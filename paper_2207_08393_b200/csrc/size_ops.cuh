@@ -76,11 +76,19 @@ inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
     static bool attr_done = false;
     cudaError_t e = ensure_smem(col_kernel<P, L, MODE>, E::SMEM_BYTES, attr_done);
     if (e != cudaSuccess) return e;
-    const long long tiles = (a.es + L - 1) / L;
+    long long tiles = (a.es + L - 1) / L;
+    ColArgs b = a;
+    if (MODE == COL_Z) {
+        // the number of sampled ranks is known only on the device: launch a bounded number of blocks
+        // per outer index and let them stride over the tiles
+        const long long cap = 4096 / (a.nouter > 0 ? a.nouter : 1) + 16;
+        if (tiles > cap) tiles = cap;
+        b.ztiles = (int)tiles;
+    }
     const long long blocks = a.nouter * tiles;
     if (blocks <= 0) return cudaSuccess;
     if (blocks > 2147483647LL) return cudaErrorInvalidConfiguration;
-    col_kernel<P, L, MODE><<<(unsigned)blocks, E::THREADS, E::SMEM_BYTES, s>>>(a);
+    col_kernel<P, L, MODE><<<(unsigned)blocks, E::THREADS, E::SMEM_BYTES, s>>>(b);
     return cudaGetLastError();
 }
 

@@ -54,8 +54,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(BUILD, "kernels_group%d.o" % g)
         jobs.append((["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) +
                      ["-DGLEAM_GROUP=%d" % g, "-c", os.path.join(CSRC, "kernels_group.cu"), "-o", obj], obj))
-    obj = os.path.join(BUILD, "gleam_dc.o")
-    jobs.append((["nvcc"] + NVCC_FLAGS + ["-c", os.path.join(CSRC, "gleam_dc.cu"), "-o", obj], obj))
+    for name in ("gleam_dc", "kernels_pairs"):
+        obj = os.path.join(BUILD, name + ".o")
+        jobs.append((["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) +
+                     ["-c", os.path.join(CSRC, name + ".cu"), "-o", obj], obj))
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4)) as ex:
         outs = list(ex.map(lambda j: _run(j[0]), jobs))
     if verbose:

@@ -12,6 +12,7 @@
 // the readout axis only; R^H y is needed at sampled positions alone.
 #include "../../include/gleam.h"
 #include "size_ops.cuh"
+#include "dc_rowtile.cuh"
 
 #include <atomic>
 #include <cmath>
@@ -24,6 +25,8 @@ namespace gleam {
 #define GLEAM_SIZE(N, A0, A1, A2, LR, B0, B1, B2, LC) extern const SizeOps size_ops_##N;
 #include "sizes.def"
 #undef GLEAM_SIZE
+
+const PairOps* find_pair(int n1, int n2);     // kernels_pairs.cu
 
 static const SizeOps* find_size(int n) {
     switch (n) {
@@ -303,8 +306,20 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
             cf* W = (cf*)(ws + L.off_W);
+            const PairOps* pair = find_pair(L.n1, L.n2);
             for (int i0 = 0; i0 < L.n0; i0 += L.G) {
                 const int g = (L.n0 - i0 < L.G) ? (L.n0 - i0) : L.G;
+                if (pair) {
+                    // row-tile kernels: every pass over the workspace is contiguous
+                    TileArgs ta{};
+                    ta.x = (const cf*)x; ta.sens = (const cf*)sens; ta.out = (cf*)out; ta.V = W; ta.mask = mask;
+                    ta.zin = z; ta.zidx = ca.zidx; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
+                    ta.C = L.C; ta.T = L.T; ta.Ts = L.Ts; ta.n0 = L.n0; ta.G = g; ta.i0_start = i0; ta.nunits = L.units;
+                    LAUNCH(GLEAM_K_ROW_FWD, pair->fwd(ta, L.images, s));
+                    LAUNCH(GLEAM_K_COL_MID_SEP, pair->mid(ta, s));
+                    LAUNCH(GLEAM_K_ROW_INV, pair->inv(ta, L.images, s));
+                    continue;
+                }
                 ra.W = W; ra.rpb = g * L.n1; ra.row0 = i0 * L.n1; ra.nrows = L.images * ra.rpb;
                 LAUNCH(GLEAM_K_ROW_FWD, op2->row(ROW_FWD, ra, s));
                 ColArgs cm = ca;

@@ -35,9 +35,9 @@ struct RowTile {
     static constexpr bool ELIGIBLE = WL::ELIGIBLE && (PZ::S == 2) && (RY % WL::LW == 0) && (RY / WL::LW <= 32);
     static constexpr int WARPS = RY / WL::LW;              // one warp per LW of the RY rows
     static constexpr int THREADS = WARPS * 32;
-    // shared memory (float2 units): tile T[RY][NZ], then per warp: S[2][LW*NZ] and the exchange area
+    // shared memory (float2 units): tile T[RY][NZ], then per warp: S[LW*NZ] and the exchange area
     static constexpr int TILE_T = RY * NZ;
-    static constexpr int PER_WARP = 2 * WL::TILE + WL::LW * WL::EXL + (WL::LW * WL::EXL) % 2;
+    static constexpr int PER_WARP = WL::TILE + WL::LW * WL::EXL + (WL::LW * WL::EXL) % 2;   // S rows (single buffer) + exchange
     static constexpr size_t SMEM_BYTES = sizeof(cf) * (TILE_T + WARPS * PER_WARP + 2);
 };
 
@@ -55,7 +55,7 @@ rowtile_kernel(const TileArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     cf* wsm = smem + RT::TILE_T + warp * RT::PER_WARP;
     cf* sS = wsm;
-    cf* sE = wsm + 2 * WL::TILE;
+    cf* sE = wsm + WL::TILE;
 
     // block -> (bt, slab gi of the chunk, j)
     const unsigned blk = blockIdx.x;
@@ -80,13 +80,24 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
     for (int k = 0; k < R0; ++k) twz[k] = unit_root_fwd<NZ>((jz * k) % NZ);
 
-    auto issue_s = [&](int c, int buf) {                     // S rows of this warp for coil c
+    // S rows of this warp for coil c.  Single buffer: the copy for the next coil is issued as soon
+    // as the warp has consumed the current one and lands while the rest of the iteration runs.
+    auto issue_s = [&](int c) {
 #pragma unroll
         for (int ll = 0; ll < LW; ++ll) {
             const long long so = __shfl_sync(0xffffffffu, s_off, ll * TPL);
             const cf* src = a.sens + so + c * s_stride;
-            for (int i = lane; i < NZ / 2; i += 32) cp_async16(sS + buf * WL::TILE + ll * NZ + 2 * i, src + 2 * i);
+            for (int i = lane; i < NZ / 2; i += 32) cp_async16(sS + ll * NZ + 2 * i, src + 2 * i);
         }
+        cp_async_commit();
+    };
+    // ky twiddles of this block's rows: w_N1^(j k0)
+    cf twy[RY];
+#pragma unroll
+    for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)j_y * k0) % N1);
+    auto v_ptr = [&](int c) -> cf* {                         // V[unit][gi][.][j][.] of coil c
+        const long long unit = ((long long)(b * a.C + c)) * a.T + t;
+        return a.V + (((unit * a.G + gi) * RY) * (long long)BY + j_y) * NZ;
     };
 
     cf xreg[R0], acc[R0];
@@ -94,26 +105,32 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
         for (int m = 0; m < R0; ++m) { xreg[m] = a.x[x_off + jz + PZ::BF0 * m]; acc[m] = make_float2(0.f, 0.f); }
     }
-    issue_s(0, 0);
-    cp_async_commit();
+    issue_s(0);
+    // pass 3: the column values of the first coil (one kz column per thread; THREADS >= NZ is not
+    // required, further columns are fetched inside the loop)
+    cf cnext[RY];
+    if (INV && (int)threadIdx.x < NZ) {
+        const cf* Vn = v_ptr(0);
+#pragma unroll
+        for (int k0 = 0; k0 < RY; ++k0) cnext[k0] = Vn[(long long)k0 * BY * NZ + threadIdx.x];
+    }
 
     for (int c = 0; c < a.C; ++c) {
-        const int buf = c & 1;
-        if (c + 1 < a.C) issue_s(c + 1, buf ^ 1);
-        cp_async_commit();
-        const long long unit = ((long long)(b * a.C + c)) * a.T + t;
-        // V[unit][gi][k0][j][kz]
-        cf* Vu = a.V + (((unit * a.G + gi) * RY) * (long long)BY + j_y) * NZ;      // + k0 * BY * NZ + kz
-        const cf* cS = sS + buf * WL::TILE + l * NZ;
+        cf* Vu = v_ptr(c);                                   // + k0 * BY * NZ + kz
+        const cf* cS = sS + l * NZ;
         cf v[R0], u[RL];
 
         if (!INV) {
-            cp_async_wait<1>();
+            cp_async_wait<0>();
             __syncwarp();
             // ---- kz transform of this warp's rows ----
             if (a0) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) v[m] = cmul(cS[jz + PZ::BF0 * m], xreg[m]);
+            }
+            __syncwarp();                                    // S rows consumed: fetch the next coil's
+            if (c + 1 < a.C) issue_s(c + 1);
+            if (a0) {
                 Dft<R0, -1>::run(v);
 #pragma unroll
                 for (int k = 0; k < R0; ++k) sE[l * WL::EXL + k * PZ::LS1 + jz] = (k == 0) ? v[0] : cmul(v[k], twz[k]);
@@ -135,7 +152,7 @@ rowtile_kernel(const TileArgs a) {
                 Dft<RY, -1>::run(cvals);
 #pragma unroll
                 for (int k0 = 0; k0 < RY; ++k0) {
-                    const cf r = (k0 == 0) ? cvals[0] : cmul(cvals[k0], unit_root_fwd<N1>(((int)j_y * k0) % N1));
+                    const cf r = (k0 == 0) ? cvals[0] : cmul(cvals[k0], twy[k0]);
                     Vu[(long long)k0 * BY * NZ + kz] = r;
                 }
             }
@@ -146,8 +163,13 @@ rowtile_kernel(const TileArgs a) {
                 cf cvals[RY];
 #pragma unroll
                 for (int k0 = 0; k0 < RY; ++k0) {
-                    const cf r = Vu[(long long)k0 * BY * NZ + kz];
-                    cvals[k0] = (k0 == 0) ? r : cmulc(r, unit_root_fwd<N1>(((int)j_y * k0) % N1));
+                    const cf r = (kz == (int)threadIdx.x) ? cnext[k0] : Vu[(long long)k0 * BY * NZ + kz];
+                    cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
+                }
+                if (kz == (int)threadIdx.x && c + 1 < a.C) {     // next coil's column, in flight during this coil
+                    const cf* Vn = v_ptr(c + 1);
+#pragma unroll
+                    for (int k0 = 0; k0 < RY; ++k0) cnext[k0] = Vn[(long long)k0 * BY * NZ + kz];
                 }
                 Dft<RY, +1>::run(cvals);
 #pragma unroll
@@ -162,7 +184,7 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
                 for (int m = 0; m < RL; ++m) sE[l * WL::EXL + jz * PZ::LS1 + m] = u[m];
             }
-            cp_async_wait<1>();
+            cp_async_wait<0>();
             __syncwarp();
             if (a0) {
 #pragma unroll
@@ -178,6 +200,8 @@ rowtile_kernel(const TileArgs a) {
                     acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
                 }
             }
+            __syncwarp();                                    // S rows consumed: fetch the next coil's
+            if (c + 1 < a.C) issue_s(c + 1);
             __syncthreads();          // tile and exchange area are reused by the next coil
         }
     }

@@ -60,7 +60,7 @@ def test_rank2_full_mask(oracle, n, weighted):
 
 
 @pytest.mark.parametrize("n", [(4, 6, 10), (2, 2, 2), (6, 10, 2), (16, 12, 20), (10, 46, 32), (32, 20, 64),
-                               (6, 64, 16), (4, 128, 24)])   # (6, 64, 16): dense weighted mask, more sampled entries per tile than the staging area
+                               (6, 64, 16), (4, 128, 24), (4, 32, 64), (6, 64, 32), (2, 320, 64)])   # (6, 64, 16): dense weighted mask, more sampled entries per tile than the staging area
 @pytest.mark.parametrize("mask_kind", [MASK_READOUT_INVARIANT, MASK_FULL])
 def test_rank3_small(oracle, n, mask_kind):
     d, x, y, sens, mask = problem(3, 2, 3, 1, n, mask_kind, weighted=(n[0] == 6), seed=sum(n) + mask_kind)

@@ -45,7 +45,7 @@ struct RowTile {
 // pass 1 (INV = false) and pass 3 (INV = true)
 // ---------------------------------------------------------------------------------------------
 template <class PZ, int RY, int BY, bool INV>
-__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS)
+__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, INV ? 1 : 2)
 rowtile_kernel(const TileArgs a) {
     using RT = RowTile<PZ, RY, BY>;
     using WL = typename RT::WL;
@@ -246,10 +246,11 @@ rowtile_mid_kernel(const TileArgs a) {
         const float mv = mk[(long long)shift_half(ky, N1) * NZ];
         c[k1] = cscale(c[k1], mv * mv * a.scale2);
         if (HAS_Z) {
-            if (mv != 0.f) {
-                const cf q = zz[zi[(long long)ky * NZ]];
-                c[k1] = make_float2(c[k1].x - q.x, c[k1].y - q.y);
-            }
+            // branch-free: unsampled entries read rank 0 and discard it
+            const int r = zi[(long long)ky * NZ];
+            const cf q = zz[r >= 0 ? r : 0];
+            const float on = (r >= 0) ? 1.f : 0.f;
+            c[k1] = make_float2(fmaf(-on, q.x, c[k1].x), fmaf(-on, q.y, c[k1].y));
         }
     }
     Dft<BY, +1>::run(c);

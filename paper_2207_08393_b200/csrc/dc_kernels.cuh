@@ -44,6 +44,7 @@ struct ColArgs {
     const int* zlist;   // (B,T,pe): sampled source positions p (unshifted), by rank
     const int* zcount;  // (B,T)
     const float* m2c;   // (B,T,pe): squared mask weight of the sampled positions, by rank
+    const int* zstart;  // row-tile path: (B,T,33) first rank of each ky-mod-RY group (null otherwise)
     const float* mask;  // COL_Z, COL_MID_SEP: readout-invariant mask; COL_MID_FULL: full mask (B,T,V)
     int es;             // element stride of the transformed axis = lines per outer index
     long long nouter;   // outer indices

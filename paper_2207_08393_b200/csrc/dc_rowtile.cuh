@@ -23,6 +23,7 @@ struct TileArgs {
     cf* V;                                    // workspace (unit, G, RY, BY, NZ)
     const float* mask;                        // (B,T,N1,NZ) readout-invariant mask (pass 2)
     const cf* zin; const int* zidx;           // compact z table and rank map (pass 2, forward call)
+    const int* zstart;                        // (B,T,33): first rank of each ky-mod-RY group
     float eta, scale2;
     int C, T, Ts, n0, G, i0_start;
     long long nunits;                         // B*C*T
@@ -221,7 +222,7 @@ __global__ void __launch_bounds__(256)
 rowtile_mid_kernel(const TileArgs a) {
     constexpr int N1 = RY * BY;
     const int kz = blockIdx.y * blockDim.x + threadIdx.x;          // gridDim.y covers NZ
-    if (kz >= NZ) return;
+    const bool col_ok = kz < NZ;
     const unsigned blk = blockIdx.x;                               // (unit, gi, k0)
     const int k0 = (int)(blk % RY);
     const unsigned gi = (blk / RY) % (unsigned)a.G;
@@ -232,10 +233,33 @@ rowtile_mid_kernel(const TileArgs a) {
     const long long bt = (long long)b * a.T + t;
     const long long pe = (long long)N1 * NZ;
     cf* Vp = a.V + ((((long long)unit * a.G + gi) * RY + k0) * BY) * NZ + kz;   // + j * NZ
+    // forward call: the z values of this block's ky group are contiguous in the compact table (ranks
+    // zstart[k0] .. zstart[k0+1]); they are staged in shared memory while the transform runs
+    constexpr int ZS_CAP = HAS_Z ? 1024 : 1;
+    __shared__ cf s_z[ZS_CAP];
+    int z_first = 0;
+    bool z_staged = false;
+    if (HAS_Z && a.zstart) {
+        z_first = a.zstart[bt * 33 + k0];
+        const int nz = a.zstart[bt * 33 + k0 + 1] - z_first;
+        z_staged = nz <= ZS_CAP;
+        if (z_staged) {
+            const cf* zsrc = a.zin + ((long long)unit * a.n0 + a.i0_start + (int)gi) * pe + z_first;
+            for (int e = threadIdx.x; e < nz; e += blockDim.x) cp_async8(&s_z[e], zsrc + e);
+            cp_async_commit();
+        }
+    }
     cf c[BY];
+    if (col_ok) {
 #pragma unroll
-    for (int j = 0; j < BY; ++j) c[j] = Vp[(long long)j * NZ];
-    Dft<BY, -1>::run(c);
+        for (int j = 0; j < BY; ++j) c[j] = Vp[(long long)j * NZ];
+        Dft<BY, -1>::run(c);
+    }
+    if (HAS_Z) {
+        cp_async_wait<0>();
+        __syncthreads();
+    }
+    if (!col_ok) return;
     const float* mk = a.mask + bt * pe + shift_half(kz, NZ);
     const int i0 = a.i0_start + (int)gi;
     const cf* zz = HAS_Z ? a.zin + ((long long)unit * a.n0 + i0) * pe : nullptr;
@@ -248,7 +272,7 @@ rowtile_mid_kernel(const TileArgs a) {
         if (HAS_Z) {
             // branch-free: unsampled entries read rank 0 and discard it
             const int r = zi[(long long)ky * NZ];
-            const cf q = zz[r >= 0 ? r : 0];
+            const cf q = z_staged ? s_z[r >= 0 ? r - z_first : 0] : zz[r >= 0 ? r : 0];
             const float on = (r >= 0) ? 1.f : 0.f;
             c[k1] = make_float2(fmaf(-on, q.x, c[k1].x), fmaf(-on, q.y, c[k1].y));
         }
@@ -262,7 +286,7 @@ rowtile_mid_kernel(const TileArgs a) {
 // launch table for the (ky, kz) pairs that have row-tile kernels
 // ---------------------------------------------------------------------------------------------
 struct PairOps {
-    int n1, n2;
+    int n1, n2, ry;
     cudaError_t (*fwd)(const TileArgs&, long long images, cudaStream_t);
     cudaError_t (*mid)(const TileArgs&, cudaStream_t);
     cudaError_t (*inv)(const TileArgs&, long long images, cudaStream_t);

@@ -46,9 +46,11 @@ static const SizeOps* find_size(int n) {
 #define ZMAP_PER_THREAD 2
 #define ZMAP_CHUNK (ZMAP_THREADS * ZMAP_PER_THREAD)
 #define ZMAP_TILE 8
+#define ZMAP_MAX_RY 32
 __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restrict__ mask, int* __restrict__ zidx,
                                                             int* __restrict__ zlist, int* __restrict__ zcount,
-                                                            float* __restrict__ m2c, int n1, int n2, int rank) {
+                                                            float* __restrict__ m2c, int* __restrict__ zstart,
+                                                            int n1, int n2, int rank, int ry) {
     __shared__ int warp_sum[ZMAP_THREADS / 32];
     __shared__ int base_sh;
     const int pe = (rank == 2) ? n2 : n1 * n2;
@@ -59,8 +61,16 @@ __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restr
     // Rank order.  rank 2: the raw k index.  rank 3: column tiles of ZMAP_TILE raw kz indices, inside
     // a tile by (raw ky, raw kz): the sampled entries that one tile of the column kernel needs are
     // then neighbours in the compact z table.  raw_of maps the scan position to the raw position.
-    const bool tiled = (rank == 3) && (n2 % ZMAP_TILE == 0);
+    // ry > 0 (row-tile path): groups of equal ky mod ry, inside a group by (ky div ry, kz): the sampled
+    // entries one block of the row-tile middle pass needs are contiguous; zstart[bt][k0] is the
+    // first rank of group k0, zstart[bt][ry] the total.
+    const bool tiled = (ry == 0) && (rank == 3) && (n2 % ZMAP_TILE == 0);
+    const int per_k0 = (ry > 0) ? (n1 / ry) * n2 : 1;
     auto raw_of = [&](int q) -> int {
+        if (ry > 0) {
+            const int k0 = q / per_k0, rem = q - k0 * per_k0;
+            return (k0 + ry * (rem / n2)) * n2 + rem % n2;
+        }
         if (!tiled) return q;
         const int per_tile = n1 * ZMAP_TILE;
         const int tile = q / per_tile, rem = q - tile * per_tile;
@@ -102,13 +112,17 @@ __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restr
     for (int e = 0; e < ZMAP_PER_THREAD; ++e) {
         const int q = q0 + e;
         if (q >= pe) break;
+        if (ry > 0 && q % per_k0 == 0) zstart[bt * (ZMAP_MAX_RY + 1) + q / per_k0] = r;
         if (on[e]) {
             const float mv = mk[src[e]];
             zidx[bt * pe + raw_of(q)] = r; zlist[bt * pe + r] = src[e]; m2c[bt * pe + r] = mv * mv; ++r;
         }
         else zidx[bt * pe + raw_of(q)] = -1;
     }
-    if (q_begin + ZMAP_CHUNK >= pe && tid == ZMAP_THREADS - 1) zcount[bt] = r;   // last chunk, last thread: total
+    if (q_begin + ZMAP_CHUNK >= pe && tid == ZMAP_THREADS - 1) {                 // last chunk, last thread: total
+        zcount[bt] = r;
+        if (ry > 0) zstart[bt * (ZMAP_MAX_RY + 1) + ry] = r;
+    }
 }
 
 static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
@@ -119,7 +133,7 @@ struct Layout {
     long long V, units, images;
     bool separable;
     // workspace (byte offsets)
-    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_m2c, off_W, total;
+    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_m2c, off_zstart, off_W, total;
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
@@ -157,7 +171,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     if (L->images * L->n0 * L->n1 >= (1ll << 31)) return GLEAM_ERR_BAD_DIMS;   // row counters are 32-bit
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
-    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_m2c = L->off_W = 0; L->G = 0;
+    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_m2c = L->off_zstart = L->off_W = 0; L->G = 0;
     if (L->separable) {
         const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
         if (with_y) {
@@ -167,6 +181,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
             L->off_zlist = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(int), 256);
             L->off_zcount = off; off = align_up(off + (uint64_t)L->images * sizeof(int), 256);
             L->off_m2c = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(float), 256);
+            L->off_zstart = off; off = align_up(off + (uint64_t)L->images * (ZMAP_MAX_RY + 1) * sizeof(int), 256);
         }
         if (L->rank == 3) {
             const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
@@ -287,11 +302,14 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             int* zlist = (int*)(ws + L.off_zlist);
             int* zcount = (int*)(ws + L.off_zcount);
             float* m2c = (float*)(ws + L.off_m2c);
+            int* zstart = (int*)(ws + L.off_zstart);
+            const PairOps* zpair = (L.rank == 3) ? find_pair(L.n1, L.n2) : nullptr;
+            const int zry = (zpair && zpair->ry <= ZMAP_MAX_RY) ? zpair->ry : 0;
             CK(prof_mark(GLEAM_K_PREP_M2, s));
             zmap_kernel<<<dim3((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images), ZMAP_THREADS, 0, s>>>(
-                mask, zidx, zlist, zcount, m2c, L.n1, L.n2, L.rank);
+                mask, zidx, zlist, zcount, m2c, zstart, L.n1, L.n2, L.rank, zry);
             CK(cudaGetLastError());
-            ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount; ca.m2c = m2c;
+            ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount; ca.m2c = m2c; ca.zstart = zry ? zstart : nullptr;
             ra.zidx = zidx;
             ColArgs cz = ca;
             cz.y = (const cf*)y; cz.z = z; cz.mask = mask;
@@ -313,7 +331,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
                     // row-tile kernels: every pass over the workspace is contiguous
                     TileArgs ta{};
                     ta.x = (const cf*)x; ta.sens = (const cf*)sens; ta.out = (cf*)out; ta.V = W; ta.mask = mask;
-                    ta.zin = z; ta.zidx = ca.zidx; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
+                    ta.zin = z; ta.zidx = ca.zidx; ta.zstart = ca.zstart; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
                     ta.C = L.C; ta.T = L.T; ta.Ts = L.Ts; ta.n0 = L.n0; ta.G = g; ta.i0_start = i0; ta.nunits = L.units;
                     LAUNCH(GLEAM_K_ROW_FWD, pair->fwd(ta, L.images, s));
                     LAUNCH(GLEAM_K_COL_MID_SEP, pair->mid(ta, s));

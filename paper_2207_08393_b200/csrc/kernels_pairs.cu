@@ -11,7 +11,7 @@ namespace gleam {
     GLEAM_PAIR(320, 16, 20, 64, 8, 8)
 
 #define GLEAM_PAIR(N1, RY, BY, N2, Z0, Z1) \
-    static const PairOps pair_##N1##_##N2 = {N1, N2, &PairImpl<Plan<N2, Z0, Z1, 1>, RY, BY>::fwd, \
+    static const PairOps pair_##N1##_##N2 = {N1, N2, RY, &PairImpl<Plan<N2, Z0, Z1, 1>, RY, BY>::fwd, \
                                              &PairImpl<Plan<N2, Z0, Z1, 1>, RY, BY>::mid,          \
                                              &PairImpl<Plan<N2, Z0, Z1, 1>, RY, BY>::inv};
 GLEAM_PAIRS

@@ -50,6 +50,7 @@ static const SizeOps* find_size(int n) {
 __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restrict__ mask, int* __restrict__ zidx,
                                                             int* __restrict__ zlist, int* __restrict__ zcount,
                                                             float* __restrict__ m2c, int* __restrict__ zstart,
+                                                            int* __restrict__ chunk_cnt, int count_only,
                                                             int n1, int n2, int rank, int ry) {
     __shared__ int warp_sum[ZMAP_THREADS / 32];
     __shared__ int base_sh;
@@ -81,13 +82,23 @@ __global__ void __launch_bounds__(ZMAP_THREADS) zmap_kernel(const float* __restr
         if (rank == 2) return shift_half(rq, n2);
         return shift_half(rq / n2, n1) * n2 + shift_half(rq % n2, n2);
     };
-    // sampled positions before this chunk
-    int c = 0;
-    for (int q = tid; q < q_begin; q += ZMAP_THREADS) c += (mk[src_of(q)] != 0.f) ? 1 : 0;
-    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-    if (lane == 0) warp_sum[warp] = c;
-    __syncthreads();
-    if (tid == 0) { int t = 0; for (int w = 0; w < ZMAP_THREADS / 32; ++w) t += warp_sum[w]; base_sh = t; }
+    // Two launches: the first (count_only) stores the number of sampled positions of every chunk,
+    // the second adds up the chunks before its own and numbers its entries.
+    const int nchunks = gridDim.x;
+    if (count_only) {
+        int c = 0;
+#pragma unroll
+        for (int e = 0; e < ZMAP_PER_THREAD; ++e) {
+            const int q = q_begin + tid * ZMAP_PER_THREAD + e;
+            c += (q < pe && mk[src_of(q)] != 0.f) ? 1 : 0;
+        }
+        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+        if (lane == 0) warp_sum[warp] = c;
+        __syncthreads();
+        if (tid == 0) { int t = 0; for (int w = 0; w < ZMAP_THREADS / 32; ++w) t += warp_sum[w]; chunk_cnt[bt * nchunks + blockIdx.x] = t; }
+        return;
+    }
+    if (tid == 0) { int t = 0; for (int w = 0; w < (int)blockIdx.x; ++w) t += chunk_cnt[bt * nchunks + w]; base_sh = t; }
     __syncthreads();
     const int base = base_sh;
     __syncthreads();
@@ -133,7 +144,7 @@ struct Layout {
     long long V, units, images;
     bool separable;
     // workspace (byte offsets)
-    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_m2c, off_zstart, off_W, total;
+    uint64_t off_z, off_zidx, off_zlist, off_zcount, off_m2c, off_zstart, off_zchunk, off_W, total;
     int G;  // readout slabs per chunk (rank 3 separable)
 };
 
@@ -171,7 +182,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     if (L->images * L->n0 * L->n1 >= (1ll << 31)) return GLEAM_ERR_BAD_DIMS;   // row counters are 32-bit
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
-    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_m2c = L->off_zstart = L->off_W = 0; L->G = 0;
+    L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_m2c = L->off_zstart = L->off_zchunk = L->off_W = 0; L->G = 0;
     if (L->separable) {
         const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
         if (with_y) {
@@ -182,6 +193,7 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
             L->off_zcount = off; off = align_up(off + (uint64_t)L->images * sizeof(int), 256);
             L->off_m2c = off; off = align_up(off + (uint64_t)L->images * pe * sizeof(float), 256);
             L->off_zstart = off; off = align_up(off + (uint64_t)L->images * (ZMAP_MAX_RY + 1) * sizeof(int), 256);
+            L->off_zchunk = off; off = align_up(off + (uint64_t)L->images * ((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK) * sizeof(int), 256);
         }
         if (L->rank == 3) {
             const uint64_t slab = (uint64_t)L->units * L->n1 * L->n2 * sizeof(cf);
@@ -306,8 +318,12 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             const PairOps* zpair = (L.rank == 3) ? find_pair(L.n1, L.n2) : nullptr;
             const int zry = (zpair && zpair->ry <= ZMAP_MAX_RY) ? zpair->ry : 0;
             CK(prof_mark(GLEAM_K_PREP_M2, s));
-            zmap_kernel<<<dim3((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images), ZMAP_THREADS, 0, s>>>(
-                mask, zidx, zlist, zcount, m2c, zstart, L.n1, L.n2, L.rank, zry);
+            int* zchunk = (int*)(ws + L.off_zchunk);
+            const dim3 zgrid((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images);
+            zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 1, L.n1, L.n2, L.rank, zry);
+            CK(cudaGetLastError());
+            CK(prof_mark(GLEAM_K_PREP_M2, s));
+            zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 0, L.n1, L.n2, L.rank, zry);
             CK(cudaGetLastError());
             ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount; ca.m2c = m2c; ca.zstart = zry ? zstart : nullptr;
             ra.zidx = zidx;

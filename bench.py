@@ -446,9 +446,10 @@ def run_ours(args, w):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # an ncu capture, keyed by (workload, kernel class); None until a capture of the current kernel exists.
 TRAFFIC = {
-    # colpipe_mid_sep_kernel<Plan<320,16,20>,8>, whole-volume launch of knee3d (1-pass ncu capture of
-    # bench.py itself, profiles/col_mid_sep_knee3d.md): forward launch 1.81 + 1.63 GB, VJP launch 1.68 + 1.62 GB
-    ("knee3d", "col_mid_sep"): 0.5 * ((1.81e9 + 1.63e9) + (1.68e9 + 1.62e9)),
+    # rowtile_kernel<Plan<256,16,16>,16,20,INV>, whole-volume launches of knee3d (1-pass ncu capture of
+    # bench.py itself, profiles/rowtile_knee3d.md): dram read + write per launch
+    ("knee3d", "row_inv"): 3.57e9 + 0.203e9,
+    ("knee3d", "row_fwd"): 1.89e9 + 1.63e9,
 }
 
 

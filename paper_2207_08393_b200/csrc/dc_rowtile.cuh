@@ -46,7 +46,7 @@ struct RowTile {
 // pass 1 (INV = false) and pass 3 (INV = true)
 // ---------------------------------------------------------------------------------------------
 template <class PZ, int RY, int BY, bool INV>
-__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, INV ? 1 : 2)
+__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, 2)
 rowtile_kernel(const TileArgs a) {
     using RT = RowTile<PZ, RY, BY>;
     using WL = typename RT::WL;
@@ -93,18 +93,29 @@ rowtile_kernel(const TileArgs a) {
         cp_async_commit();
     };
     // ky twiddles of this block's rows: w_N1^(j k0)
-    cf twy[RY];
+    // (pass 3 keeps them in shared memory: they are the same for the whole block, and the registers
+    // are needed for the coil sum)
+    cf twy[INV ? 1 : RY];
+    __shared__ cf s_twy[INV ? RY : 1];
+    if (INV) {
+        if ((int)threadIdx.x < RY) s_twy[threadIdx.x] = unit_root_fwd<N1>(((int)j_y * (int)threadIdx.x) % N1);
+        __syncthreads();
+    } else {
 #pragma unroll
-    for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)j_y * k0) % N1);
+        for (int k0 = 0; k0 < RY; ++k0) twy[INV ? 0 : k0] = unit_root_fwd<N1>(((int)j_y * k0) % N1);
+    }
     auto v_ptr = [&](int c) -> cf* {                         // V[unit][gi][.][j][.] of coil c
         const long long unit = ((long long)(b * a.C + c)) * a.T + t;
         return a.V + (((unit * a.G + gi) * RY) * (long long)BY + j_y) * NZ;
     };
 
-    cf xreg[R0], acc[R0];
-    if (a0) {
+    cf xreg[INV ? 1 : R0], acc[INV ? R0 : 1];      // pass 1 keeps x, pass 3 the coil sum (and reads x at the end)
+    if (INV) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) { xreg[m] = a.x[x_off + jz + PZ::BF0 * m]; acc[m] = make_float2(0.f, 0.f); }
+        for (int m = 0; m < R0; ++m) acc[INV ? m : 0] = make_float2(0.f, 0.f);
+    } else if (a0) {
+#pragma unroll
+        for (int m = 0; m < R0; ++m) xreg[INV ? 0 : m] = a.x[x_off + jz + PZ::BF0 * m];
     }
     issue_s(0);
     // pass 3: the column values of the first coil (one kz column per thread; THREADS >= NZ is not
@@ -127,7 +138,7 @@ rowtile_kernel(const TileArgs a) {
             // ---- kz transform of this warp's rows ----
             if (a0) {
 #pragma unroll
-                for (int m = 0; m < R0; ++m) v[m] = cmul(cS[jz + PZ::BF0 * m], xreg[m]);
+                for (int m = 0; m < R0; ++m) v[m] = cmul(cS[jz + PZ::BF0 * m], xreg[INV ? 0 : m]);
             }
             __syncwarp();                                    // S rows consumed: fetch the next coil's
             if (c + 1 < a.C) issue_s(c + 1);
@@ -153,7 +164,7 @@ rowtile_kernel(const TileArgs a) {
                 Dft<RY, -1>::run(cvals);
 #pragma unroll
                 for (int k0 = 0; k0 < RY; ++k0) {
-                    const cf r = (k0 == 0) ? cvals[0] : cmul(cvals[k0], twy[k0]);
+                    const cf r = (k0 == 0) ? cvals[0] : cmul(cvals[k0], twy[INV ? 0 : k0]);
                     Vu[(long long)k0 * BY * NZ + kz] = r;
                 }
             }
@@ -165,7 +176,7 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
                 for (int k0 = 0; k0 < RY; ++k0) {
                     const cf r = (kz == (int)threadIdx.x) ? cnext[k0] : Vu[(long long)k0 * BY * NZ + kz];
-                    cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
+                    cvals[k0] = (k0 == 0) ? r : cmulc(r, s_twy[INV ? k0 : 0]);
                 }
                 if (kz == (int)threadIdx.x && c + 1 < a.C) {     // next coil's column, in flight during this coil
                     const cf* Vn = v_ptr(c + 1);
@@ -197,8 +208,9 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
                     const cf sv = cS[jz + PZ::BF0 * m];
-                    acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
-                    acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
+                    cf& am = acc[INV ? m : 0];
+                    am.x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, am.x));
+                    am.y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, am.y));
                 }
             }
             __syncwarp();                                    // S rows consumed: fetch the next coil's
@@ -209,8 +221,11 @@ rowtile_kernel(const TileArgs a) {
     cp_async_wait<0>();
     if (INV && a0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m)
-            a.out[x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y));
+        for (int m = 0; m < R0; ++m) {
+            const cf xv = a.x[x_off + jz + PZ::BF0 * m];
+            const cf am = acc[INV ? m : 0];
+            a.out[x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, am.x, xv.x), fmaf(-a.eta, am.y, xv.y));
+        }
     }
 }
 

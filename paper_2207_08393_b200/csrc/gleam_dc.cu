@@ -320,9 +320,11 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
             CK(prof_mark(GLEAM_K_PREP_M2, s));
             int* zchunk = (int*)(ws + L.off_zchunk);
             const dim3 zgrid((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images);
-            zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 1, L.n1, L.n2, L.rank, zry);
-            CK(cudaGetLastError());
-            CK(prof_mark(GLEAM_K_PREP_M2, s));
+            if (zgrid.x > 1) {        // a table of one chunk needs no counts of earlier chunks
+                zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 1, L.n1, L.n2, L.rank, zry);
+                CK(cudaGetLastError());
+                CK(prof_mark(GLEAM_K_PREP_M2, s));
+            }
             zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 0, L.n1, L.n2, L.rank, zry);
             CK(cudaGetLastError());
             ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount; ca.m2c = m2c; ca.zstart = zry ? zstart : nullptr;

@@ -1,6 +1,6 @@
 """Small, seeded invocation of the data-consistency step for profiler captures.
 
-    python -m paper_2207_08393_b200.profile_case knee3d_small    # 8 coils, 20x320x256 (3 workspace chunks)
+    python -m paper_2207_08393_b200.profile_case knee3d_small    # 8 coils, 20x320x256
     python -m paper_2207_08393_b200.profile_case cine            # 8 coils, 20 frames of 192x160
 
 Runs three forward + VJP pairs through the C ABI on random inputs of the workload's shape and

@@ -23,6 +23,7 @@ struct TileArgs {
     cf* V;                                    // workspace (unit, G, RY, BY, NZ)
     const float* mask;                        // (B,T,N1,NZ) readout-invariant mask (pass 2)
     const cf* zin; const int* zidx;           // compact z table and rank map (pass 2, forward call)
+    const float* m2c;                         // squared mask weights by rank (pass 2, forward call)
     const int* zstart;                        // (B,T,33): first rank of each ky-mod-RY group
     float eta, scale2;
     int C, T, Ts, n0, G, i0_start;
@@ -46,7 +47,7 @@ struct RowTile {
 // pass 1 (INV = false) and pass 3 (INV = true)
 // ---------------------------------------------------------------------------------------------
 template <class PZ, int RY, int BY, bool INV>
-__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, 2)
+__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, INV ? 1 : 2)
 rowtile_kernel(const TileArgs a) {
     using RT = RowTile<PZ, RY, BY>;
     using WL = typename RT::WL;
@@ -93,29 +94,18 @@ rowtile_kernel(const TileArgs a) {
         cp_async_commit();
     };
     // ky twiddles of this block's rows: w_N1^(j k0)
-    // (pass 3 keeps them in shared memory: they are the same for the whole block, and the registers
-    // are needed for the coil sum)
-    cf twy[INV ? 1 : RY];
-    __shared__ cf s_twy[INV ? RY : 1];
-    if (INV) {
-        if ((int)threadIdx.x < RY) s_twy[threadIdx.x] = unit_root_fwd<N1>(((int)j_y * (int)threadIdx.x) % N1);
-        __syncthreads();
-    } else {
+    cf twy[RY];
 #pragma unroll
-        for (int k0 = 0; k0 < RY; ++k0) twy[INV ? 0 : k0] = unit_root_fwd<N1>(((int)j_y * k0) % N1);
-    }
+    for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)j_y * k0) % N1);
     auto v_ptr = [&](int c) -> cf* {                         // V[unit][gi][.][j][.] of coil c
         const long long unit = ((long long)(b * a.C + c)) * a.T + t;
         return a.V + (((unit * a.G + gi) * RY) * (long long)BY + j_y) * NZ;
     };
 
-    cf xreg[INV ? 1 : R0], acc[INV ? R0 : 1];      // pass 1 keeps x, pass 3 the coil sum (and reads x at the end)
-    if (INV) {
+    cf xreg[R0], acc[R0];
+    if (a0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) acc[INV ? m : 0] = make_float2(0.f, 0.f);
-    } else if (a0) {
-#pragma unroll
-        for (int m = 0; m < R0; ++m) xreg[INV ? 0 : m] = a.x[x_off + jz + PZ::BF0 * m];
+        for (int m = 0; m < R0; ++m) { xreg[m] = a.x[x_off + jz + PZ::BF0 * m]; acc[m] = make_float2(0.f, 0.f); }
     }
     issue_s(0);
     // pass 3: the column values of the first coil (one kz column per thread; THREADS >= NZ is not
@@ -138,7 +128,7 @@ rowtile_kernel(const TileArgs a) {
             // ---- kz transform of this warp's rows ----
             if (a0) {
 #pragma unroll
-                for (int m = 0; m < R0; ++m) v[m] = cmul(cS[jz + PZ::BF0 * m], xreg[INV ? 0 : m]);
+                for (int m = 0; m < R0; ++m) v[m] = cmul(cS[jz + PZ::BF0 * m], xreg[m]);
             }
             __syncwarp();                                    // S rows consumed: fetch the next coil's
             if (c + 1 < a.C) issue_s(c + 1);
@@ -164,7 +154,7 @@ rowtile_kernel(const TileArgs a) {
                 Dft<RY, -1>::run(cvals);
 #pragma unroll
                 for (int k0 = 0; k0 < RY; ++k0) {
-                    const cf r = (k0 == 0) ? cvals[0] : cmul(cvals[k0], twy[INV ? 0 : k0]);
+                    const cf r = (k0 == 0) ? cvals[0] : cmul(cvals[k0], twy[k0]);
                     Vu[(long long)k0 * BY * NZ + kz] = r;
                 }
             }
@@ -176,7 +166,7 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
                 for (int k0 = 0; k0 < RY; ++k0) {
                     const cf r = (kz == (int)threadIdx.x) ? cnext[k0] : Vu[(long long)k0 * BY * NZ + kz];
-                    cvals[k0] = (k0 == 0) ? r : cmulc(r, s_twy[INV ? k0 : 0]);
+                    cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
                 }
                 if (kz == (int)threadIdx.x && c + 1 < a.C) {     // next coil's column, in flight during this coil
                     const cf* Vn = v_ptr(c + 1);
@@ -208,9 +198,8 @@ rowtile_kernel(const TileArgs a) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
                     const cf sv = cS[jz + PZ::BF0 * m];
-                    cf& am = acc[INV ? m : 0];
-                    am.x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, am.x));
-                    am.y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, am.y));
+                    acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
+                    acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
                 }
             }
             __syncwarp();                                    // S rows consumed: fetch the next coil's
@@ -221,11 +210,8 @@ rowtile_kernel(const TileArgs a) {
     cp_async_wait<0>();
     if (INV && a0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) {
-            const cf xv = a.x[x_off + jz + PZ::BF0 * m];
-            const cf am = acc[INV ? m : 0];
-            a.out[x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, am.x, xv.x), fmaf(-a.eta, am.y, xv.y));
-        }
+        for (int m = 0; m < R0; ++m)
+            a.out[x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y));
     }
 }
 
@@ -250,8 +236,10 @@ rowtile_mid_kernel(const TileArgs a) {
     cf* Vp = a.V + ((((long long)unit * a.G + gi) * RY + k0) * BY) * NZ + kz;   // + j * NZ
     // forward call: the z values of this block's ky group are contiguous in the compact table (ranks
     // zstart[k0] .. zstart[k0+1]); they are staged in shared memory while the transform runs
+    // with their scaled squared mask weights; slot ZS_CAP holds zero for the unsampled entries
     constexpr int ZS_CAP = HAS_Z ? 1024 : 1;
-    __shared__ cf s_z[ZS_CAP];
+    __shared__ cf s_z[ZS_CAP + 1];
+    __shared__ float s_w[ZS_CAP + 1];
     int z_first = 0;
     bool z_staged = false;
     if (HAS_Z && a.zstart) {
@@ -260,8 +248,11 @@ rowtile_mid_kernel(const TileArgs a) {
         z_staged = nz <= ZS_CAP;
         if (z_staged) {
             const cf* zsrc = a.zin + ((long long)unit * a.n0 + a.i0_start + (int)gi) * pe + z_first;
+            const float* wsrc = a.m2c + bt * pe + z_first;
             for (int e = threadIdx.x; e < nz; e += blockDim.x) cp_async8(&s_z[e], zsrc + e);
             cp_async_commit();
+            for (int e = threadIdx.x; e < nz; e += blockDim.x) s_w[e] = wsrc[e] * a.scale2;
+            if (threadIdx.x == 0) { s_z[ZS_CAP] = make_float2(0.f, 0.f); s_w[ZS_CAP] = 0.f; }
         }
     }
     cf c[BY];
@@ -279,17 +270,31 @@ rowtile_mid_kernel(const TileArgs a) {
     const int i0 = a.i0_start + (int)gi;
     const cf* zz = HAS_Z ? a.zin + ((long long)unit * a.n0 + i0) * pe : nullptr;
     const int* zi = HAS_Z ? a.zidx + bt * pe + kz : nullptr;
+    const float* m2 = HAS_Z ? a.m2c + bt * pe : nullptr;
+    if (HAS_Z && z_staged) {
+        // forward call: weight and z value by rank from shared memory, branch-free (unsampled
+        // entries point at the zero slot)
 #pragma unroll
-    for (int k1 = 0; k1 < BY; ++k1) {
-        const int ky = k0 + RY * k1;                                // raw k index along ky
-        const float mv = mk[(long long)shift_half(ky, N1) * NZ];
-        c[k1] = cscale(c[k1], mv * mv * a.scale2);
-        if (HAS_Z) {
-            // branch-free: unsampled entries read rank 0 and discard it
-            const int r = zi[(long long)ky * NZ];
-            const cf q = z_staged ? s_z[r >= 0 ? r - z_first : 0] : zz[r >= 0 ? r : 0];
-            const float on = (r >= 0) ? 1.f : 0.f;
-            c[k1] = make_float2(fmaf(-on, q.x, c[k1].x), fmaf(-on, q.y, c[k1].y));
+        for (int k1 = 0; k1 < BY; ++k1) {
+            const int r = zi[(long long)(k0 + RY * k1) * NZ];
+            const int e = (r >= 0) ? r - z_first : ZS_CAP;
+            const float w = s_w[e];
+            const cf q = s_z[e];
+            c[k1] = make_float2(fmaf(w, c[k1].x, -q.x), fmaf(w, c[k1].y, -q.y));
+        }
+    } else {
+#pragma unroll
+        for (int k1 = 0; k1 < BY; ++k1) {
+            const int ky = k0 + RY * k1;                            // raw k index along ky
+            if (HAS_Z) {                                            // more sampled entries than the staging area holds
+                const int r = zi[(long long)ky * NZ];
+                const float w = (r >= 0) ? m2[r] * a.scale2 : 0.f;
+                const cf q = (r >= 0) ? zz[r] : make_float2(0.f, 0.f);
+                c[k1] = make_float2(fmaf(w, c[k1].x, -q.x), fmaf(w, c[k1].y, -q.y));
+            } else {
+                const float mv = mk[(long long)shift_half(ky, N1) * NZ];
+                c[k1] = cscale(c[k1], mv * mv * a.scale2);
+            }
         }
     }
     Dft<BY, +1>::run(c);

@@ -349,7 +349,7 @@ static int run(const void* x, const void* y, const void* sens, const float* mask
                     // row-tile kernels: every pass over the workspace is contiguous
                     TileArgs ta{};
                     ta.x = (const cf*)x; ta.sens = (const cf*)sens; ta.out = (cf*)out; ta.V = W; ta.mask = mask;
-                    ta.zin = z; ta.zidx = ca.zidx; ta.zstart = ca.zstart; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
+                    ta.zin = z; ta.zidx = ca.zidx; ta.m2c = ca.m2c; ta.zstart = ca.zstart; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
                     ta.C = L.C; ta.T = L.T; ta.Ts = L.Ts; ta.n0 = L.n0; ta.G = g; ta.i0_start = i0; ta.nunits = L.units;
                     LAUNCH(GLEAM_K_ROW_FWD, pair->fwd(ta, L.images, s));
                     LAUNCH(GLEAM_K_COL_MID_SEP, pair->mid(ta, s));

@@ -29,6 +29,10 @@
  *
  * Inputs are single precision (the arrays the GPU sees), promoted to double; outputs are double.
  *
+ * The MoDL model inversion of Eq. 7 by conjugate gradients is further down (oracle_modl_cg); its
+ * pins are in tests/test_oracle_modl.py (closed form for A^H A = I, dense solve, Krylov-space
+ * minimiser for the truncated iteration).
+ *
  * Pins (tests/test_oracle_pins.py): brute-force DFT, closed-form spectra of deltas and
  * constants, Parseval, adjoint identity, Hermitian/PSD normal operator, A^H A = I for a full mask
  * and unit-norm sensitivities, affine structure, an independent library FFT.
@@ -396,6 +400,161 @@ int oracle_dc(const float* x, const float* y, const float* sens, const float* ma
             }
         }
     free(contrib);
+    return rc;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * MoDL data-consistency step (the model inversion of Eq. 7, second line):
+ *
+ *      x = (A^H A + mu I)^{-1} (A^H y + mu z)
+ *
+ * solved, as the paper states, with the conjugate gradient method and a fixed number of steps
+ * (10 in its experiments).  The paper prints no CG listing; this is the textbook method of
+ * Hestenes and Stiefel for the Hermitian positive definite system H x = b, H = A^H A + mu I,
+ * with the choices the paper leaves open fixed as follows: start at x_0 = 0 (so r_0 = p_0 = b),
+ * no preconditioner, exactly n_iter steps, stop early only when the residual is exactly zero,
+ * one system per batch example (its frames solved jointly).
+ *
+ *      alpha_k = <r_k, r_k> / <p_k, H p_k>        x_{k+1} = x_k + alpha_k p_k
+ *      r_{k+1} = r_k - alpha_k H p_k              beta_k  = <r_{k+1}, r_{k+1}> / <r_k, r_k>
+ *      p_{k+1} = r_{k+1} + beta_k p_k
+ * ------------------------------------------------------------------------------------------ */
+
+/* out = A^H A p for a double-precision image p (B,T,V): S_c .* p, F, M .* M, F^H, conj(S_c), coil sum */
+static int normal_op(const zc* p, const float* sens, const float* mask, const odims* o, zc* kwork,
+                     zc* out, int nthreads)
+{
+    int rc = ORACLE_OK;
+    const int64_t units = o->B * o->C * o->T;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel for num_threads(nthreads) schedule(dynamic, 1)
+#endif
+    for (int64_t u = 0; u < units; ++u) {
+        const int64_t t = u % o->T, c = (u / o->T) % o->C, b = u / (o->T * o->C);
+        const zc* ps = p + (b * o->T + t) * o->V;
+        const float* ss = sens_ptr(sens, o, b, c, t);
+        zc* ku = kwork + u * o->V;
+        for (int64_t q = 0; q < o->V; ++q) ku[q] = ((double)ss[2 * q] + I * (double)ss[2 * q + 1]) * ps[q];
+        int r = fft_centered_volume(ku, o->n, o->rank, -1);
+        for (int64_t q = 0; q < o->V; ++q) {
+            const double m = mask_at(mask, o, b, t, q);
+            ku[q] = m * (m * ku[q]);
+        }
+        if (r == ORACLE_OK) r = fft_centered_volume(ku, o->n, o->rank, +1);
+        for (int64_t q = 0; q < o->V; ++q) ku[q] = conj((double)ss[2 * q] + I * (double)ss[2 * q + 1]) * ku[q];
+        if (r != ORACLE_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            rc = r;
+        }
+    }
+    for (int64_t b = 0; b < o->B; ++b)
+        for (int64_t t = 0; t < o->T; ++t) {
+            zc* dst = out + (b * o->T + t) * o->V;
+            for (int64_t q = 0; q < o->V; ++q) dst[q] = 0.0;
+            for (int64_t c = 0; c < o->C; ++c) {
+                const zc* src = kwork + ((b * o->C + c) * o->T + t) * o->V;
+                for (int64_t q = 0; q < o->V; ++q) dst[q] += src[q];
+            }
+        }
+    return rc;
+}
+
+/* out = A^H A p  (exported for the pins: the dense matrix of H is assembled from it) */
+int oracle_normal_op(const zc* p, const float* sens, const float* mask, const int64_t* dims, zc* out, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK || !p || !sens || !mask || !out) return ORACLE_ERR_ARG;
+    zc* kwork = (zc*)malloc(sizeof(zc) * (size_t)(o.B * o.C * o.T * o.V));
+    if (!kwork) return ORACLE_ERR_MEM;
+    const int rc = normal_op(p, sens, mask, &o, kwork, out, nthreads);
+    free(kwork);
+    return rc;
+}
+
+/* n_iter CG steps on (A^H A + mu I) x = b from x = 0.  b is overwritten (it becomes the residual).
+ * Every batch example is its own system (A is block diagonal over the batch): the inner products,
+ * alpha and beta are taken per example, over its frames and voxels, so a result does not depend
+ * on what else is in the batch.  An example whose residual is exactly zero is left as it is. */
+static int cg_solve(zc* b, const float* sens, const float* mask, const odims* o, double mu, int n_iter,
+                    zc* x, int nthreads)
+{
+    const int64_t ne = o->T * o->V;              /* elements of one example */
+    const int64_t n = o->B * ne;
+    zc* p = (zc*)malloc(sizeof(zc) * (size_t)n);
+    zc* Hp = (zc*)malloc(sizeof(zc) * (size_t)n);
+    zc* kwork = (zc*)malloc(sizeof(zc) * (size_t)(o->B * o->C * o->T * o->V));
+    double* rr = (double*)malloc(sizeof(double) * (size_t)o->B);
+    if (!p || !Hp || !kwork || !rr) { free(p); free(Hp); free(kwork); free(rr); return ORACLE_ERR_MEM; }
+    int rc = ORACLE_OK;
+    zc* r = b;
+    for (int64_t e = 0; e < o->B; ++e) {
+        rr[e] = 0.0;
+        for (int64_t i = e * ne; i < (e + 1) * ne; ++i) {
+            x[i] = 0.0; p[i] = r[i];
+            rr[e] += creal(r[i]) * creal(r[i]) + cimag(r[i]) * cimag(r[i]);
+        }
+    }
+    for (int k = 0; k < n_iter && rc == ORACLE_OK; ++k) {
+        rc = normal_op(p, sens, mask, o, kwork, Hp, nthreads);
+        for (int64_t e = 0; e < o->B; ++e) {
+            if (!(rr[e] > 0.0)) continue;
+            double pHp = 0.0;
+            for (int64_t i = e * ne; i < (e + 1) * ne; ++i) {
+                Hp[i] += mu * p[i];
+                pHp += creal(conj(p[i]) * Hp[i]);
+            }
+            const double alpha = rr[e] / pHp;
+            double rr_new = 0.0;
+            for (int64_t i = e * ne; i < (e + 1) * ne; ++i) {
+                x[i] += alpha * p[i];
+                r[i] -= alpha * Hp[i];
+                rr_new += creal(r[i]) * creal(r[i]) + cimag(r[i]) * cimag(r[i]);
+            }
+            const double beta = rr_new / rr[e];
+            for (int64_t i = e * ne; i < (e + 1) * ne; ++i) p[i] = r[i] + beta * p[i];
+            rr[e] = rr_new;
+        }
+    }
+    free(p); free(Hp); free(kwork); free(rr);
+    return rc;
+}
+
+/* x = (A^H A + mu I)^{-1} (A^H y + mu z) by n_iter CG steps (Eq. 7).  z: image (B,T,V), y: k-space. */
+int oracle_modl_cg(const float* z, const float* y, const float* sens, const float* mask, double mu, int n_iter,
+                   const int64_t* dims, zc* out, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK || !z || !y || !sens || !mask || !out || n_iter < 0) return ORACLE_ERR_ARG;
+    const int64_t n = o.B * o.T * o.V, nk = o.B * o.C * o.T * o.V;
+    zc* b = (zc*)malloc(sizeof(zc) * (size_t)n);
+    zc* k = (zc*)malloc(sizeof(zc) * (size_t)nk);
+    if (!b || !k) { free(b); free(k); return ORACLE_ERR_MEM; }
+    for (int64_t i = 0; i < nk; ++i) k[i] = (double)y[2 * i] + I * (double)y[2 * i + 1];
+    int rc = oracle_apply_AH(k, sens, mask, dims, b, nthreads);          /* b = A^H y */
+    free(k);
+    for (int64_t i = 0; i < n; ++i) b[i] += mu * ((double)z[2 * i] + I * (double)z[2 * i + 1]);
+    if (rc == ORACLE_OK) rc = cg_solve(b, sens, mask, &o, mu, n_iter, out, nthreads);
+    free(b);
+    return rc;
+}
+
+/* Vector-Jacobian product of the step with respect to z, the CG solve taken as the exact inverse
+ * (x = H^{-1}(A^H y + mu z), H Hermitian  =>  grad_z = mu H^{-1} g), evaluated by the same number
+ * of CG steps:  n_iter steps on H u = mu g  from u = 0. */
+int oracle_modl_cg_vjp(const float* g, const float* sens, const float* mask, double mu, int n_iter,
+                       const int64_t* dims, zc* out, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK || !g || !sens || !mask || !out || n_iter < 0) return ORACLE_ERR_ARG;
+    const int64_t n = o.B * o.T * o.V;
+    zc* b = (zc*)malloc(sizeof(zc) * (size_t)n);
+    if (!b) return ORACLE_ERR_MEM;
+    for (int64_t i = 0; i < n; ++i) b[i] = mu * ((double)g[2 * i] + I * (double)g[2 * i + 1]);
+    const int rc = cg_solve(b, sens, mask, &o, mu, n_iter, out, nthreads);
+    free(b);
     return rc;
 }
 

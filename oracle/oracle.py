@@ -52,6 +52,12 @@ def _load():
         lib.oracle_apply_AH.restype = i32
         lib.oracle_dc.argtypes = [p, p, p, p, dbl, p, p, i32]
         lib.oracle_dc.restype = i32
+        lib.oracle_normal_op.argtypes = [p, p, p, p, p, i32]
+        lib.oracle_normal_op.restype = i32
+        lib.oracle_modl_cg.argtypes = [p, p, p, p, dbl, i32, p, p, i32]
+        lib.oracle_modl_cg.restype = i32
+        lib.oracle_modl_cg_vjp.argtypes = [p, p, p, dbl, i32, p, p, i32]
+        lib.oracle_modl_cg_vjp.restype = i32
         lib.oracle_max_threads.argtypes = []
         lib.oracle_max_threads.restype = i32
         _lib = lib
@@ -198,5 +204,39 @@ def dc_vjp(g, sens, mask, eta: float, d: Dims, nthreads: int = 1) -> np.ndarray:
     out = np.empty(d.image_shape(), dtype=np.complex128)
     dd = d.as_array()
     rc = _load().oracle_dc(_ptr(g), None, _ptr(sens), _ptr(mask), float(eta), _ptr(dd), _ptr(out), nthreads)
+    assert rc == 0, rc
+    return out
+
+
+def normal_op(p, sens, mask, d: Dims, nthreads: int = 1) -> np.ndarray:
+    """A^H A p for a double-precision image p."""
+    p = np.ascontiguousarray(np.asarray(p, dtype=np.complex128).reshape(d.image_shape()))
+    sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
+    out = np.empty(d.image_shape(), dtype=np.complex128)
+    dd = d.as_array()
+    rc = _load().oracle_normal_op(_ptr(p), _ptr(sens), _ptr(mask), _ptr(dd), _ptr(out), nthreads)
+    assert rc == 0, rc
+    return out
+
+
+def modl_cg_forward(z, y, sens, mask, mu: float, n_iter: int, d: Dims, nthreads: int = 1) -> np.ndarray:
+    """Eq. 7: x = (A^H A + mu I)^{-1} (A^H y + mu z) by n_iter conjugate-gradient steps from zero."""
+    z = _c64(z, d.image_shape()); y = _c64(y, d.kspace_shape())
+    sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
+    out = np.empty(d.image_shape(), dtype=np.complex128)
+    dd = d.as_array()
+    rc = _load().oracle_modl_cg(_ptr(z), _ptr(y), _ptr(sens), _ptr(mask), float(mu), int(n_iter), _ptr(dd),
+                                _ptr(out), nthreads)
+    assert rc == 0, rc
+    return out
+
+
+def modl_cg_vjp(g, sens, mask, mu: float, n_iter: int, d: Dims, nthreads: int = 1) -> np.ndarray:
+    """grad_z = mu (A^H A + mu I)^{-1} g by n_iter conjugate-gradient steps from zero."""
+    g = _c64(g, d.image_shape()); sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
+    out = np.empty(d.image_shape(), dtype=np.complex128)
+    dd = d.as_array()
+    rc = _load().oracle_modl_cg_vjp(_ptr(g), _ptr(sens), _ptr(mask), float(mu), int(n_iter), _ptr(dd), _ptr(out),
+                                    nthreads)
     assert rc == 0, rc
     return out

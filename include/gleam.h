@@ -157,6 +157,34 @@ GLEAM_API int gleam_dc_forward_static(const void* x, const void* y, const void* 
                                       void* out, const gleam_dims* dims);
 GLEAM_API uint64_t gleam_dc_static_scratch_bytes(void);
 
+/* ---- MoDL data-consistency step (Eq. 7, second line) -------------------------------------------
+ *
+ *     out = (A^H A + mu I)^{-1} (A^H y + mu z)
+ *
+ * by n_iter conjugate-gradient steps (the paper's experiments use 10), A = Omega F S as above.  The
+ * paper prints no CG listing; the choices it leaves open are fixed as: start from zero, no
+ * preconditioner, exactly n_iter steps, one system per batch example (inner products over the
+ * example's frames and voxels, so a result does not depend on the rest of the batch), an example
+ * whose residual is exactly zero is left as it is.
+ *
+ *   z, out   : device, complex64 (B,T,n0,n1,n2); out == z (exact alias) is allowed
+ *   y, sens, mask, dims : as for gleam_dc_forward
+ *   mu       : > 0 (GLEAM_ERR_BAD_DIMS otherwise); n_iter in [0, 1000]; n_iter = 0 gives out = 0
+ *   dims->workspace: gleam_modl_cg_workspace_size bytes (the data-consistency workspace, three
+ *              image-sized vectors and the reduction scratch)
+ *
+ * gleam_modl_cg_vjp is the vector-Jacobian product with respect to z with the solve taken as the
+ * exact inverse (the Jacobian mu (A^H A + mu I)^{-1} is Hermitian):
+ *     grad_z = mu (A^H A + mu I)^{-1} grad_out     by n_iter conjugate-gradient steps from zero.
+ * Inner products are accumulated in double precision in a fixed order: results are deterministic.
+ * Everything is enqueued on dims->stream; no allocation, no synchronisation.
+ */
+GLEAM_API int gleam_modl_cg_forward(const void* z, const void* y, const void* sens, const float* mask, float mu,
+                                    int32_t n_iter, void* out, const gleam_dims* dims);
+GLEAM_API int gleam_modl_cg_vjp(const void* grad_out, const void* sens, const float* mask, float mu,
+                                int32_t n_iter, void* grad_z, const gleam_dims* dims);
+GLEAM_API int gleam_modl_cg_workspace_size(const gleam_dims* dims, uint64_t* bytes);
+
 /*
  * Measurement aids (no counterpart in the paper).
  * gleam_dc_launch_count: kernels this library has launched since it was loaded.
@@ -175,7 +203,8 @@ enum {
     GLEAM_K_COL_MID_FULL = 6, /* same as 4 for a full mask */
     GLEAM_K_COL_FWD = 7,
     GLEAM_K_COL_INV = 8,
-    GLEAM_K_CLASSES = 9
+    GLEAM_K_CG_VEC = 9,       /* image-sized vector kernels of the conjugate-gradient solve */
+    GLEAM_K_CLASSES = 10
 };
 GLEAM_API uint64_t gleam_dc_launch_count(void);
 GLEAM_API int gleam_dc_profile_begin(void);

@@ -1,5 +1,5 @@
 """B200-native multi-coil SENSE data-consistency step (GLEAM, arXiv 2207.08393, Eq. 3) and its
-vector-Jacobian product.  The arithmetic lives in the CUDA library ``libgleam_dc.so`` (C ABI in
+vector-Jacobian product, plus the MoDL model inversion (Eq. 7) by conjugate gradients.  The arithmetic lives in the CUDA library ``libgleam_dc.so`` (C ABI in
 ``include/gleam.h``); this package is the argument-marshalling binding plus the seeded synthetic
 workload generators."""
 from . import workloads  # noqa: F401
@@ -8,4 +8,5 @@ from .binding import (  # noqa: F401
     gleam_dc_length_supported, gleam_dc_vjp, gleam_dc_workspace_size, gleam_dims, gleam_status_string,
     gleam_version, load_library, make_dims, gleam_dc_forward_host, gleam_dc_vjp_host, gleam_dc_host_arena_size,
     gleam_dc_forward_static, gleam_dc_static_scratch_bytes, gleam_dc_launch_count, gleam_dc_profile_begin, gleam_dc_profile_end, KERNEL_CLASSES,
+    ModlCG, gleam_modl_cg_forward, gleam_modl_cg_vjp, gleam_modl_cg_workspace_size,
 )

@@ -30,10 +30,11 @@ GLEAM_MASK_READOUT_INVARIANT = 1
 EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam_dc_length_supported",
            "gleam_status_string", "gleam_version", "gleam_dc_forward_host", "gleam_dc_vjp_host",
            "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end",
-           "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes"]
+           "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes",
+           "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size"]
 
 KERNEL_CLASSES = ["zmap", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
-                  "col_inv"]
+                  "col_inv", "cg_vec"]
 
 
 class gleam_dims(ctypes.Structure):
@@ -95,6 +96,12 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_dc_forward_static.restype = i32
         lib.gleam_dc_static_scratch_bytes.argtypes = []
         lib.gleam_dc_static_scratch_bytes.restype = u64
+        lib.gleam_modl_cg_forward.argtypes = [vp, vp, vp, vp, f32, ctypes.c_int32, vp, dp]
+        lib.gleam_modl_cg_forward.restype = i32
+        lib.gleam_modl_cg_vjp.argtypes = [vp, vp, vp, f32, ctypes.c_int32, vp, dp]
+        lib.gleam_modl_cg_vjp.restype = i32
+        lib.gleam_modl_cg_workspace_size.argtypes = [dp, ctypes.POINTER(u64)]
+        lib.gleam_modl_cg_workspace_size.restype = i32
         lib.gleam_dc_launch_count.argtypes = []
         lib.gleam_dc_launch_count.restype = u64
         lib.gleam_dc_profile_begin.argtypes = []
@@ -249,3 +256,44 @@ class DataConsistency:
             grad_in = self._torch.empty_like(grad_out)
         gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, self.dims())
         return grad_in
+
+
+def gleam_modl_cg_workspace_size(dims: gleam_dims) -> int:
+    out = ctypes.c_uint64(0)
+    _check(load_library().gleam_modl_cg_workspace_size(ctypes.byref(dims), ctypes.byref(out)))
+    return int(out.value)
+
+
+def gleam_modl_cg_forward(z, y, sens, mask, mu, n_iter, out, dims: gleam_dims) -> None:
+    """out = (A^H A + mu I)^{-1} (A^H y + mu z) by n_iter conjugate-gradient steps (Eq. 7)."""
+    _check(load_library().gleam_modl_cg_forward(_addr(z), _addr(y), _addr(sens), _addr(mask), float(mu), int(n_iter),
+                                                 _addr(out), ctypes.byref(dims)))
+
+
+def gleam_modl_cg_vjp(grad_out, sens, mask, mu, n_iter, grad_z, dims: gleam_dims) -> None:
+    """grad_z = mu (A^H A + mu I)^{-1} grad_out by n_iter conjugate-gradient steps."""
+    _check(load_library().gleam_modl_cg_vjp(_addr(grad_out), _addr(sens), _addr(mask), float(mu), int(n_iter),
+                                             _addr(grad_z), ctypes.byref(dims)))
+
+
+class ModlCG(DataConsistency):
+    """Holder of dims + workspace for the MoDL model inversion of one problem shape."""
+
+    def __init__(self, batch, coils, frames, fft_rank, n, sens_has_frames=0,
+                 mask_kind=GLEAM_MASK_READOUT_INVARIANT, stream=None):
+        super().__init__(batch, coils, frames, fft_rank, n, sens_has_frames, mask_kind, stream)
+        probe = make_dims(batch, coils, frames, fft_rank, n, sens_has_frames, mask_kind)
+        nbytes = gleam_modl_cg_workspace_size(probe)
+        self.workspace = self._torch.empty(max(nbytes, 256), dtype=self._torch.uint8, device="cuda")
+
+    def solve(self, z, y, sens, mask, mu, n_iter=10, out=None):
+        if out is None:
+            out = self._torch.empty_like(z)
+        gleam_modl_cg_forward(z, y, sens, mask, mu, n_iter, out, self.dims())
+        return out
+
+    def solve_vjp(self, grad_out, sens, mask, mu, n_iter=10, grad_z=None):
+        if grad_z is None:
+            grad_z = self._torch.empty_like(grad_out)
+        gleam_modl_cg_vjp(grad_out, sens, mask, mu, n_iter, grad_z, self.dims())
+        return grad_z

@@ -1,0 +1,19 @@
+// Entry points of the data-consistency path that other translation units of the library use.
+#pragma once
+#include <cuda_runtime.h>
+#include "../../include/gleam.h"
+
+namespace gleam {
+
+// out = x - eta A^H (A x - y)   (y == nullptr: out = x - eta A^H A x).  Validates its arguments,
+// enqueues on d->stream, returns GLEAM_OK or a GLEAM_ERR_* code.
+int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
+        const gleam_dims* d);
+
+// GLEAM_OK for a device (or managed) pointer, GLEAM_ERR_NOT_DEVICE_POINTER otherwise
+int check_device_ptr(const void* p);
+
+// counts a launch of kernel class cls and, while per-kernel timing is on, records its event
+cudaError_t prof_mark(int cls, cudaStream_t s);
+
+}  // namespace gleam

@@ -13,6 +13,7 @@
 #include "../../include/gleam.h"
 #include "size_ops.cuh"
 #include "dc_rowtile.cuh"
+#include "dc_entry.h"
 
 #include <atomic>
 #include <cmath>
@@ -216,7 +217,7 @@ static bool check_pointers_enabled() {
     return v == 1;
 }
 
-static int check_device_ptr(const void* p) {
+int check_device_ptr(const void* p) {
     if (!check_pointers_enabled()) return GLEAM_OK;
     cudaPointerAttributes at;
     cudaError_t e = cudaPointerGetAttributes(&at, p);
@@ -242,7 +243,7 @@ static std::vector<cudaEvent_t> g_prof_events;   // event i is recorded just bef
 static std::vector<int> g_prof_class;            // kernel class of launch i, -1 = end-of-call marker
 static size_t g_prof_used = 0;
 
-static cudaError_t prof_mark(int cls, cudaStream_t s) {
+cudaError_t prof_mark(int cls, cudaStream_t s) {
     if (cls >= 0) g_launches.fetch_add(1, std::memory_order_relaxed);
     if (!g_prof_on) return cudaSuccess;
     std::lock_guard<std::mutex> lock(g_prof_mutex);
@@ -258,8 +259,8 @@ static cudaError_t prof_mark(int cls, cudaStream_t s) {
 }
 #define LAUNCH(cls, call) do { CK(prof_mark((cls), s)); CK(call); } while (0)
 
-static int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-               const gleam_dims* d) {
+int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
+        const gleam_dims* d) {
     if (!d) return GLEAM_ERR_NULL_POINTER;
     if (!x || !sens || !mask || !out) return GLEAM_ERR_NULL_POINTER;
     Layout L;

@@ -48,3 +48,31 @@ def assert_close(got, ref, x_in, what=""):
     assert rel <= REL_L2_TOL, "%s: rel L2 %.3e > %.1e" % (what, rel, REL_L2_TOL)
     assert mab <= MAX_ABS_TOL, "%s: max abs %.3e > %.1e (units of max|x|)" % (what, mab, MAX_ABS_TOL)
     return rel, mab
+
+
+def run_gpu_modl(z, y, sens, mask, mu, n_iter, fft_rank, sens_has_frames, mask_kind, in_place=False):
+    """MoDL model inversion (y given) or its VJP (y None) through the C ABI.  Returns complex64 numpy."""
+    import torch
+    import paper_2207_08393_b200 as g
+    dev = torch.device("cuda:0")
+    B, T = z.shape[0], z.shape[1]
+    C = sens.shape[1]
+    n = z.shape[2:]
+    tz = torch.from_numpy(np.ascontiguousarray(z, dtype=np.complex64)).to(dev)
+    ts = torch.from_numpy(np.ascontiguousarray(sens, dtype=np.complex64)).to(dev)
+    tm = torch.from_numpy(np.ascontiguousarray(mask, dtype=np.float32)).to(dev)
+    ty = None if y is None else torch.from_numpy(np.ascontiguousarray(y, dtype=np.complex64)).to(dev)
+    probe = g.make_dims(B, C, T, fft_rank, n, sens_has_frames, mask_kind)
+    nbytes = g.gleam_modl_cg_workspace_size(probe)
+    ws = torch.empty(nbytes + 512, dtype=torch.uint8, device=dev)
+    ws[nbytes:] = 0xA5                                   # canary behind the workspace
+    out = tz if in_place else torch.full_like(tz, float("nan"))
+    d = g.make_dims(B, C, T, fft_rank, n, sens_has_frames, mask_kind, stream=torch.cuda.current_stream(),
+                    workspace=ws.data_ptr(), workspace_bytes=nbytes)
+    if ty is not None:
+        g.gleam_modl_cg_forward(tz, ty, ts, tm, mu, n_iter, out, d)
+    else:
+        g.gleam_modl_cg_vjp(tz, ts, tm, mu, n_iter, out, d)
+    torch.cuda.synchronize()
+    assert bool((ws[nbytes:] == 0xA5).all()), "workspace overrun"
+    return out.cpu().numpy()

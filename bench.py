@@ -87,6 +87,8 @@ def kernel_work(cls, w, launches_per_call):
         return W * 24, W * (10 * l2(nro) + 6)
     if cls in ("col_fwd", "col_inv"):
         return W * 16, W * (5 * l2(w.n[1]))
+    if cls == "cg_vec":         # image-sized vector kernels of the CG solve: on average 3.7 passes of 8 B
+        return W * (3.7 * 8 / C), W * (8.0 / C)     # per voxel (init 5, dot 2, step 6, dir 3 passes)
     return 0.0, 0.0
 
 
@@ -443,6 +445,185 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+MODL_METRIC = "modl_cg_solve_plus_vjp_throughput"
+
+
+def run_modl(args, w):
+    """MoDL model inversion (Eq. 7): one step = gleam_modl_cg_forward + gleam_modl_cg_vjp, each with
+    --cg-steps conjugate-gradient steps.  `value` counts voxel*coils per application of the normal
+    operator A^H A (the solve applies it cg_steps + 1 times counting the right-hand side A^H y, the
+    VJP cg_steps times), so it is comparable with the data-consistency metric."""
+    import numpy as np
+    import torch
+    n_iter, mu = args.cg_steps, args.mu
+    ops_per_step = 2 * n_iter + 1
+    if args.impl == "reference":
+        rank, world, _ = dist_setup(args.gpus)
+        if rank != 0:
+            return
+        from oracle import oracle
+        oracle.build()
+        ws, sample_txt = reference_sample(w)
+        inp, y = make_problem(ws)
+        d = oracle.Dims(ws.batch, ws.coils, ws.frames, ws.fft_rank, ws.n, 0, oracle.MASK_READOUT_INVARIANT)
+        cores = oracle.max_threads()
+        for _ in range(args.warmup):
+            oracle.modl_cg_forward(inp["x"], y, inp["sens"], inp["mask"], mu, 1, d, nthreads=cores)
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            oracle.modl_cg_forward(inp["x"], y, inp["sens"], inp["mask"], mu, n_iter, d, nthreads=cores)
+            oracle.modl_cg_vjp(inp["g"], inp["sens"], inp["mask"], mu, n_iter, d, nthreads=cores)
+        dt = time.perf_counter() - t0
+        value = ws.voxel_coils * ops_per_step * args.steps / dt
+        print(json.dumps({
+            "impl": "reference", "metric": MODL_METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "description": w.description, "sample": sample_txt, "mu": mu, "cg_steps": n_iter},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample_txt},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+        return
+
+    import paper_2207_08393_b200 as g
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    g.load_library()
+    peaks = load_peaks()
+    inp, y = make_problem(w, seed_offset=rank)
+    tz, tg, ts, tm, ty = (torch.from_numpy(a).to(dev) for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
+    cg = g.ModlCG(w.batch, w.coils, w.frames, w.fft_rank, w.n)
+    out, gz = torch.empty_like(tz), torch.empty_like(tg)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        cg.solve(tz, ty, ts, tm, mu, n_iter, out)
+        cg.solve_vjp(tg, ts, tm, mu, n_iter, gz)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)       # L2 is 126 MB
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3 if sampler else 0.0)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    launches0 = g.gleam_dc_launch_count()
+    t_begin = time.time()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for a, b in evs:
+        flush.fill_(1)
+        a.record(stream)
+        step()
+        b.record(stream)
+    barrier()
+    local_ms = sum(a.elapsed_time(b) for a, b in evs)
+    launches = g.gleam_dc_launch_count() - launches0
+    t_end = time.time()
+    total_ms, total_units = aggregate(local_ms, w.voxel_coils * ops_per_step * args.steps, world, dist, dev)
+    value = total_units / (total_ms * 1e-3)
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
+
+    # ---- per-kernel pass (CUDA events around every launch) -------------------------------------
+    prof_steps = min(args.steps, 3)
+    g.gleam_dc_profile_begin()
+    for _ in range(prof_steps):
+        flush.fill_(1)
+        step()
+    prof = g.gleam_dc_profile_end()
+    kernels = {}
+    for cls, (ms, cnt) in prof.items():
+        nbytes, flops = kernel_work(cls, w, 1.0)         # every launch covers the whole problem
+        avg_s = ms * 1e-3 / cnt
+        kernels[cls] = {"launches_per_step": cnt / prof_steps, "ms_per_step": ms / prof_steps, "avg_us": avg_s * 1e6,
+                        "gbs": nbytes / avg_s / 1e9, "tflops": flops / avg_s / 1e12}
+
+    # ---- end to end: pinned host inputs copied in, results copied out, every step ----------------
+    e2e_steps = max(1, min(args.steps, 5))
+    hz, hg, hs, hm, hy = (torch.from_numpy(a).pin_memory() for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
+    hout, hgz = torch.empty_like(hz).pin_memory(), torch.empty_like(hg).pin_memory()
+
+    def step_host():
+        dz, dg, ds, dm, dy = (t.to(dev, non_blocking=True) for t in (hz, hg, hs, hm, hy))
+        cg.solve(dz, dy, ds, dm, mu, n_iter, out)
+        cg.solve_vjp(dg, ds, dm, mu, n_iter, gz)
+        hout.copy_(out, non_blocking=True)
+        hgz.copy_(gz, non_blocking=True)
+
+    step_host()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        step_host()
+    e1.record(stream)
+    barrier()
+    e2e_ms, e2e_units = aggregate(e0.elapsed_time(e1), w.voxel_coils * ops_per_step * e2e_steps, world, dist, dev)
+    nb = lambda t: t.numel() * t.element_size()
+    h2d, d2h = sum(nb(t) for t in (hz, hg, hs, hm, hy)), nb(hout) + nb(hgz)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    alu_peak = fp32_peak_tflops(peaks["sm_max_mhz"])
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    kd = kernels[dom]
+    t_hbm, t_alu = kd["gbs"] / peaks["hbm_gbs"], kd["tflops"] / alu_peak
+    if t_hbm >= t_alu:
+        roof = {"bound": "hbm", "achieved": kd["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": t_hbm}
+    else:
+        roof = {"bound": "alu", "achieved": kd["tflops"], "peak": alu_peak, "unit": "TFLOP/s", "frac": t_alu}
+    roof.update({"kernel": dom, "peak_source": peaks["source"] + (" copy bandwidth" if roof["bound"] == "hbm" else
+                 " sm_max_mhz x 148 SMs x 128 lanes x 2"), "traffic": None,
+                 "share_of_step": kd["ms_per_step"] / sum(k["ms_per_step"] for k in kernels.values())})
+    # whole step against the operator's own roofline: ops_per_step applications of A^H A at their VJP bound
+    nbytes, flops = call_roofline(w, False)
+    bound_s = ops_per_step * max(nbytes / (peaks["hbm_gbs"] * 1e9), flops / (alu_peak * 1e12))
+    step_roof = {"operator_applications": ops_per_step, "bound_us": bound_s * 1e6,
+                 "measured_us": total_ms / args.steps * 1e3, "frac": bound_s / (total_ms / args.steps * 1e-3)}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import oracle
+        oracle.build()
+        cores = oracle.max_threads()
+        wsamp, sample_txt = reference_sample(w)
+        inp_c, y_c = (inp, y) if wsamp is w else make_problem(wsamp)
+        d = oracle.Dims(wsamp.batch, wsamp.coils, wsamp.frames, wsamp.fft_rank, wsamp.n, 0, oracle.MASK_READOUT_INVARIANT)
+        t0 = time.perf_counter()
+        oracle.modl_cg_forward(inp_c["x"], y_c, inp_c["sens"], inp_c["mask"], mu, n_iter, d, nthreads=cores)
+        oracle.modl_cg_vjp(inp_c["g"], inp_c["sens"], inp_c["mask"], mu, n_iter, d, nthreads=cores)
+        dt = time.perf_counter() - t0
+        cpu = {"value": wsamp.voxel_coils * ops_per_step / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": sample_txt + ", 1 step", "seconds": dt}
+
+    print(json.dumps({
+        "metric": MODL_METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "description": w.description, "mu": mu, "cg_steps": n_iter,
+                   "step": "1 gleam_modl_cg_forward + 1 gleam_modl_cg_vjp; value counts voxel*coils per application "
+                           "of A^H A (%d per step)" % ops_per_step,
+                   "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "256 MB L2 flush before every step"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(launches), "roofline": roof, "step_roofline": step_roof, "kernels": kernels, "cpu_baseline": cpu}))
+    if dist is not None:
+        dist.destroy_process_group()
+
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # an ncu capture, keyed by (workload, kernel class); None until a capture of the current kernel exists.
 TRAFFIC = {
@@ -461,10 +642,17 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="knee3d")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--method", default="dc", choices=["dc", "modl"],
+                    help="dc: the gradient data-consistency step (Eq. 3); modl: the model inversion of Eq. 7 "
+                         "by 10 conjugate-gradient steps (use with --workload knee2d or cine)")
+    ap.add_argument("--mu", type=float, default=0.05)
+    ap.add_argument("--cg-steps", type=int, default=10)
     args = ap.parse_args()
     from paper_2207_08393_b200 import workloads as wl
     w = wl.WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.method == "modl":
+        run_modl(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

@@ -216,6 +216,175 @@ rowtile_kernel(const TileArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// pass 3, persistent form: one block per SM walks over the (b,t,slab,j) items with stride gridDim.x
+// and keeps its loads one step ahead across item boundaries: while the last coil of an item is
+// processed, the sensitivity rows and the workspace column of the next item's first coil are
+// already in flight, and the x rows of an item arrive (cp.async into shared memory) while its coils
+// are summed.  At one block per SM nothing else would hide the start-up latency of an item.
+// ---------------------------------------------------------------------------------------------
+template <class PZ, int RY, int BY>
+struct RowTileInv {
+    using RT = RowTile<PZ, RY, BY>;
+    using WL = typename RT::WL;
+    static constexpr int XROWS = WL::LW * PZ::N;                         // x rows of one warp
+    static constexpr int PER_WARP = RT::PER_WARP + XROWS;
+    static constexpr size_t SMEM_BYTES = sizeof(cf) * (RT::TILE_T + RT::WARPS * PER_WARP + 2);
+};
+
+template <class PZ, int RY, int BY>
+__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, 1)
+rowtile_inv_kernel(const TileArgs a, const unsigned nitems) {
+    using RT = RowTile<PZ, RY, BY>;
+    using RI = RowTileInv<PZ, RY, BY>;
+    using WL = typename RT::WL;
+    constexpr int NZ = PZ::N, R0 = PZ::R0, RL = PZ::RL, TPL = WL::TPL, LW = WL::LW, N1 = RY * BY;
+    extern __shared__ __align__(16) float2 smem[];
+    cf* sT = smem;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    cf* wsm = smem + RT::TILE_T + warp * RI::PER_WARP;
+    cf* sS = wsm;
+    cf* sE = wsm + WL::TILE;
+    cf* sX = wsm + RT::PER_WARP;
+
+    const int l = lane / TPL, jz = lane % TPL;
+    const int m_row = warp * LW + l;                         // 0 .. RY-1
+    const bool a0 = jz < PZ::BF0, aL = jz < PZ::BFL;
+    const long long V3 = (long long)a.n0 * N1 * NZ;
+    const long long s_stride = (long long)a.Ts * V3;
+
+    struct Item { unsigned j_y, gi; int b, t; long long x_off, s_off; };
+    auto decode = [&](unsigned item) -> Item {
+        Item it;
+        it.j_y = item % BY;
+        it.gi = (item / BY) % (unsigned)a.G;
+        const unsigned bt = item / (BY * (unsigned)a.G);
+        it.b = (int)(bt / (unsigned)a.T);
+        it.t = (int)(bt - (unsigned)it.b * a.T);
+        const int ky = (int)it.j_y + BY * m_row;             // image-side row of this lane
+        const long long row_elems = ((long long)(a.i0_start + (int)it.gi) * N1 + ky) * NZ;
+        it.x_off = (long long)bt * V3 + row_elems;
+        it.s_off = ((long long)(it.b * a.C) * a.Ts + (a.Ts > 1 ? it.t : 0)) * V3 + row_elems;
+        return it;
+    };
+    auto v_ptr = [&](const Item& it, int c) -> const cf* {   // V[unit][gi][.][j][.] of coil c
+        const long long unit = ((long long)(it.b * a.C + c)) * a.T + it.t;
+        return a.V + (((unit * a.G + it.gi) * RY) * (long long)BY + it.j_y) * NZ;
+    };
+    auto issue_s = [&](const Item& it, int c) {              // S rows of this warp -> sS (one commit group)
+#pragma unroll
+        for (int ll = 0; ll < LW; ++ll) {
+            const long long so = __shfl_sync(0xffffffffu, it.s_off, ll * TPL);
+            const cf* src = a.sens + so + c * s_stride;
+            for (int i = lane; i < NZ / 2; i += 32) cp_async16(sS + ll * NZ + 2 * i, src + 2 * i);
+        }
+        cp_async_commit();
+    };
+    auto issue_x = [&](const Item& it) {                     // x rows of this warp -> sX (one commit group)
+#pragma unroll
+        for (int ll = 0; ll < LW; ++ll) {
+            const long long xo = __shfl_sync(0xffffffffu, it.x_off, ll * TPL);
+            for (int i = lane; i < NZ / 2; i += 32) cp_async16(sX + ll * NZ + 2 * i, a.x + xo + 2 * i);
+        }
+        cp_async_commit();
+    };
+
+    cf twz[R0];                                              // kz inter-stage twiddles of this lane
+#pragma unroll
+    for (int k = 0; k < R0; ++k) twz[k] = unit_root_fwd<NZ>((jz * k) % NZ);
+
+    unsigned item = blockIdx.x;
+    if (item >= nitems) return;
+    Item cur = decode(item);
+    issue_s(cur, 0);
+    cf cnext[RY];                                            // workspace column of the coming coil
+    if ((int)threadIdx.x < NZ) {
+        const cf* Vn = v_ptr(cur, 0);
+#pragma unroll
+        for (int k0 = 0; k0 < RY; ++k0) cnext[k0] = Vn[(long long)k0 * BY * NZ + threadIdx.x];
+    }
+
+    for (;;) {
+        const unsigned nxt = item + gridDim.x;
+        const bool has_next = nxt < nitems;                  // the same in every thread of the block
+        const Item nx = decode(has_next ? nxt : item);
+        issue_x(cur);                                        // newest commit group during the first coil
+        cf twy[RY];                                          // ky twiddles of this item's rows: w_N1^(j k0)
+#pragma unroll
+        for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)cur.j_y * k0) % N1);
+        cf acc[R0];
+#pragma unroll
+        for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
+
+        for (int c = 0; c < a.C; ++c) {
+            const cf* Vu = v_ptr(cur, c);
+            const cf* cS = sS + l * NZ;
+            cf v[R0], u[RL];
+            // ---- inverse radix-RY across the rows, one kz column per thread ----
+            for (int kz = threadIdx.x; kz < NZ; kz += RT::THREADS) {
+                cf cvals[RY];
+#pragma unroll
+                for (int k0 = 0; k0 < RY; ++k0) {
+                    const cf r = (kz == (int)threadIdx.x) ? cnext[k0] : Vu[(long long)k0 * BY * NZ + kz];
+                    cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
+                }
+                if (kz == (int)threadIdx.x && (c + 1 < a.C || has_next)) {   // the coming coil's column
+                    const cf* Vn = (c + 1 < a.C) ? v_ptr(cur, c + 1) : v_ptr(nx, 0);
+#pragma unroll
+                    for (int k0 = 0; k0 < RY; ++k0) cnext[k0] = Vn[(long long)k0 * BY * NZ + kz];
+                }
+                Dft<RY, +1>::run(cvals);
+#pragma unroll
+                for (int m = 0; m < RY; ++m) sT[m * NZ + kz] = cvals[m];
+            }
+            __syncthreads();
+            // ---- kz inverse of this warp's rows, conjugate-sensitivity coil sum ----
+            if (aL) {
+#pragma unroll
+                for (int k = 0; k < RL; ++k) u[k] = sT[m_row * NZ + jz + PZ::BFL * k];
+                Dft<RL, +1>::run(u);
+#pragma unroll
+                for (int m = 0; m < RL; ++m) sE[l * WL::EXL + jz * PZ::LS1 + m] = u[m];
+            }
+            // S rows of this coil have landed; during the first coil the x rows may stay in flight
+            if (c == 0) cp_async_wait<1>(); else cp_async_wait<0>();
+            __syncwarp();
+            if (a0) {
+#pragma unroll
+                for (int k = 0; k < R0; ++k) {
+                    const cf r = sE[l * WL::EXL + k * PZ::LS1 + jz];
+                    v[k] = (k == 0) ? r : cmulc(r, twz[k]);
+                }
+                Dft<R0, +1>::run(v);
+#pragma unroll
+                for (int m = 0; m < R0; ++m) {
+                    const cf sv = cS[jz + PZ::BF0 * m];
+                    acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
+                    acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
+                }
+            }
+            __syncwarp();                                    // S rows consumed: fetch the coming coil's
+            if (c + 1 < a.C) issue_s(cur, c + 1);
+            else if (has_next) issue_s(nx, 0);
+            __syncthreads();          // tile and exchange area are reused by the next coil
+        }
+        // ---- update: the x rows are complete once everything but the newest group has landed ----
+        if (has_next) cp_async_wait<1>(); else cp_async_wait<0>();
+        __syncwarp();
+        if (a0) {
+#pragma unroll
+            for (int m = 0; m < R0; ++m) {
+                const cf xv = sX[l * NZ + jz + PZ::BF0 * m];
+                a.out[cur.x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
+            }
+        }
+        __syncwarp();                                        // x rows read: the next item may overwrite them
+        if (!has_next) break;
+        item = nxt;
+        cur = nx;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // pass 2: radix-BY transform over j, mask and z, inverse; one kz column per thread, no shared memory
 // ---------------------------------------------------------------------------------------------
 template <int NZ, int RY, int BY, bool HAS_Z>
@@ -327,7 +496,24 @@ struct PairImpl {
         return cudaGetLastError();
     }
     static cudaError_t fwd(const TileArgs& a, long long images, cudaStream_t s) { return rows<false>(a, images, s); }
-    static cudaError_t inv(const TileArgs& a, long long images, cudaStream_t s) { return rows<true>(a, images, s); }
+    static cudaError_t inv(const TileArgs& a, long long images, cudaStream_t s) {
+        using RI = RowTileInv<PZ, RY, BY>;
+        static bool done = false;
+        cudaError_t e = ensure_smem(rowtile_inv_kernel<PZ, RY, BY>, RI::SMEM_BYTES, done);
+        if (e != cudaSuccess) return e;
+        const long long items = images * a.G * BY;
+        if (items <= 0) return cudaSuccess;
+        if (items > 2147483647LL) return cudaErrorInvalidConfiguration;
+        static int sms = 0;                                   // one persistent block per SM
+        if (sms == 0) {
+            int dev = 0;
+            if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+            if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        }
+        const unsigned grid = (unsigned)(items < sms ? items : sms);
+        rowtile_inv_kernel<PZ, RY, BY><<<grid, RT::THREADS, RI::SMEM_BYTES, s>>>(a, (unsigned)items);
+        return cudaGetLastError();
+    }
     static cudaError_t mid(const TileArgs& a, cudaStream_t s) {
         constexpr int NZ = PZ::N;
         const int threads = NZ < 256 ? ((NZ + 31) / 32) * 32 : 256;

@@ -216,19 +216,25 @@ rowtile_kernel(const TileArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// pass 3, persistent form: one block per SM walks over the (b,t,slab,j) items with stride gridDim.x
-// and keeps its loads one step ahead across item boundaries: while the last coil of an item is
-// processed, the sensitivity rows and the workspace column of the next item's first coil are
-// already in flight, and the x rows of an item arrive (cp.async into shared memory) while its coils
-// are summed.  At one block per SM nothing else would hide the start-up latency of an item.
+// pass 3, persistent form: one block per SM walks over its (b,t,slab,j) items and their coils as
+// one flat sequence of steps s = (item, coil) and keeps the loads of two steps in flight: the
+// workspace columns V(s) and the sensitivity rows S(s) arrive by cp.async in double-buffered
+// shared memory, and the copies for step s+2 are issued as soon as step s has consumed its
+// buffer, across item boundaries.  At one block per SM (the coil sum, x and both twiddle sets live
+// in registers) one step of loads in flight does not cover the memory latency.
+// Commit groups are issued in the fixed order V(0) S(0) V(1) S(1) | V(s+2) S(s+2) per step, empty
+// where the sequence has ended, so that "all but the newest three" is always the wait that a
+// consumer needs.
 // ---------------------------------------------------------------------------------------------
 template <class PZ, int RY, int BY>
 struct RowTileInv {
     using RT = RowTile<PZ, RY, BY>;
     using WL = typename RT::WL;
-    static constexpr int XROWS = WL::LW * PZ::N;                         // x rows of one warp
-    static constexpr int PER_WARP = RT::PER_WARP + XROWS;
-    static constexpr size_t SMEM_BYTES = sizeof(cf) * (RT::TILE_T + RT::WARPS * PER_WARP + 2);
+    static constexpr int TILE_V = RY * PZ::N;                            // one workspace column set
+    static constexpr int PER_WARP = RT::PER_WARP + WL::TILE;             // second buffer of S rows
+    static constexpr int OFF_V = RT::TILE_T;
+    static constexpr int OFF_WARP = RT::TILE_T + 2 * TILE_V;
+    static constexpr size_t SMEM_BYTES = sizeof(cf) * (OFF_WARP + RT::WARPS * PER_WARP + 2);
 };
 
 template <class PZ, int RY, int BY>
@@ -240,20 +246,25 @@ rowtile_inv_kernel(const TileArgs a, const unsigned nitems) {
     constexpr int NZ = PZ::N, R0 = PZ::R0, RL = PZ::RL, TPL = WL::TPL, LW = WL::LW, N1 = RY * BY;
     extern __shared__ __align__(16) float2 smem[];
     cf* sT = smem;
+    cf* sV = smem + RI::OFF_V;                               // [2][RY][NZ]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    cf* wsm = smem + RT::TILE_T + warp * RI::PER_WARP;
-    cf* sS = wsm;
-    cf* sE = wsm + WL::TILE;
-    cf* sX = wsm + RT::PER_WARP;
+    cf* wsm = smem + RI::OFF_WARP + warp * RI::PER_WARP;
+    cf* sS = wsm;                                            // [2][LW][NZ]
+    cf* sE = wsm + 2 * WL::TILE;
 
     const int l = lane / TPL, jz = lane % TPL;
     const int m_row = warp * LW + l;                         // 0 .. RY-1
     const bool a0 = jz < PZ::BF0, aL = jz < PZ::BFL;
     const long long V3 = (long long)a.n0 * N1 * NZ;
     const long long s_stride = (long long)a.Ts * V3;
+    const unsigned C = (unsigned)a.C;
+    if (blockIdx.x >= nitems) return;
+    const unsigned my_items = (nitems - blockIdx.x + gridDim.x - 1) / gridDim.x;
+    const unsigned total = my_items * C;                     // steps of this block (host: items * C < 2^32)
 
     struct Item { unsigned j_y, gi; int b, t; long long x_off, s_off; };
-    auto decode = [&](unsigned item) -> Item {
+    auto decode = [&](unsigned step) -> Item {               // item of step s = (s / C)-th item of this block
+        const unsigned item = blockIdx.x + (step / C) * gridDim.x;
         Item it;
         it.j_y = item % BY;
         it.gi = (item / BY) % (unsigned)a.G;
@@ -266,24 +277,31 @@ rowtile_inv_kernel(const TileArgs a, const unsigned nitems) {
         it.s_off = ((long long)(it.b * a.C) * a.Ts + (a.Ts > 1 ? it.t : 0)) * V3 + row_elems;
         return it;
     };
-    auto v_ptr = [&](const Item& it, int c) -> const cf* {   // V[unit][gi][.][j][.] of coil c
-        const long long unit = ((long long)(it.b * a.C + c)) * a.T + it.t;
-        return a.V + (((unit * a.G + it.gi) * RY) * (long long)BY + it.j_y) * NZ;
-    };
-    auto issue_s = [&](const Item& it, int c) {              // S rows of this warp -> sS (one commit group)
-#pragma unroll
-        for (int ll = 0; ll < LW; ++ll) {
-            const long long so = __shfl_sync(0xffffffffu, it.s_off, ll * TPL);
-            const cf* src = a.sens + so + c * s_stride;
-            for (int i = lane; i < NZ / 2; i += 32) cp_async16(sS + ll * NZ + 2 * i, src + 2 * i);
+    // workspace columns of step s -> sV[s & 1]: V[unit][gi][k0][j][kz], all RY rows k0 (one commit group)
+    auto issue_v = [&](unsigned step) {
+        if (step < total) {
+            const Item it = decode(step);
+            const long long unit = ((long long)(it.b * a.C + (int)(step % C))) * a.T + it.t;
+            const cf* src = a.V + (((unit * a.G + it.gi) * RY) * (long long)BY + it.j_y) * NZ;
+            cf* dst = sV + (step & 1) * RI::TILE_V;
+            for (int i = threadIdx.x; i < RY * (NZ / 2); i += RT::THREADS) {
+                const int k0 = i / (NZ / 2), part = i - k0 * (NZ / 2);
+                cp_async16(dst + k0 * NZ + 2 * part, src + (long long)k0 * BY * NZ + 2 * part);
+            }
         }
         cp_async_commit();
     };
-    auto issue_x = [&](const Item& it) {                     // x rows of this warp -> sX (one commit group)
+    // sensitivity rows of this warp for step s -> sS[s & 1] (one commit group)
+    auto issue_s = [&](unsigned step) {
+        if (step < total) {
+            const Item it = decode(step);
+            cf* dst = sS + (step & 1) * WL::TILE;
 #pragma unroll
-        for (int ll = 0; ll < LW; ++ll) {
-            const long long xo = __shfl_sync(0xffffffffu, it.x_off, ll * TPL);
-            for (int i = lane; i < NZ / 2; i += 32) cp_async16(sX + ll * NZ + 2 * i, a.x + xo + 2 * i);
+            for (int ll = 0; ll < LW; ++ll) {
+                const long long so = __shfl_sync(0xffffffffu, it.s_off, ll * TPL);
+                const cf* src = a.sens + so + (long long)(step % C) * s_stride;
+                for (int i = lane; i < NZ / 2; i += 32) cp_async16(dst + ll * NZ + 2 * i, src + 2 * i);
+            }
         }
         cp_async_commit();
     };
@@ -292,96 +310,78 @@ rowtile_inv_kernel(const TileArgs a, const unsigned nitems) {
 #pragma unroll
     for (int k = 0; k < R0; ++k) twz[k] = unit_root_fwd<NZ>((jz * k) % NZ);
 
-    unsigned item = blockIdx.x;
-    if (item >= nitems) return;
-    Item cur = decode(item);
-    issue_s(cur, 0);
-    cf cnext[RY];                                            // workspace column of the coming coil
-    if ((int)threadIdx.x < NZ) {
-        const cf* Vn = v_ptr(cur, 0);
-#pragma unroll
-        for (int k0 = 0; k0 < RY; ++k0) cnext[k0] = Vn[(long long)k0 * BY * NZ + threadIdx.x];
-    }
+    issue_v(0); issue_s(0); issue_v(1); issue_s(1);
+    cp_async_wait<3>();                                      // V(0)
+    __syncthreads();
 
-    for (;;) {
-        const unsigned nxt = item + gridDim.x;
-        const bool has_next = nxt < nitems;                  // the same in every thread of the block
-        const Item nx = decode(has_next ? nxt : item);
-        issue_x(cur);                                        // newest commit group during the first coil
-        cf twy[RY];                                          // ky twiddles of this item's rows: w_N1^(j k0)
+    Item cur = decode(0);
+    cf twy[RY], xreg[R0], acc[R0];
+    for (unsigned step = 0; step < total; ++step) {
+        const unsigned c = step % C;
+        if (c == 0) {                                        // a new item: its rows of x, its ky twiddles
+            cur = decode(step);
 #pragma unroll
-        for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)cur.j_y * k0) % N1);
-        cf acc[R0];
-#pragma unroll
-        for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
-
-        for (int c = 0; c < a.C; ++c) {
-            const cf* Vu = v_ptr(cur, c);
-            const cf* cS = sS + l * NZ;
-            cf v[R0], u[RL];
-            // ---- inverse radix-RY across the rows, one kz column per thread ----
-            for (int kz = threadIdx.x; kz < NZ; kz += RT::THREADS) {
-                cf cvals[RY];
-#pragma unroll
-                for (int k0 = 0; k0 < RY; ++k0) {
-                    const cf r = (kz == (int)threadIdx.x) ? cnext[k0] : Vu[(long long)k0 * BY * NZ + kz];
-                    cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
-                }
-                if (kz == (int)threadIdx.x && (c + 1 < a.C || has_next)) {   // the coming coil's column
-                    const cf* Vn = (c + 1 < a.C) ? v_ptr(cur, c + 1) : v_ptr(nx, 0);
-#pragma unroll
-                    for (int k0 = 0; k0 < RY; ++k0) cnext[k0] = Vn[(long long)k0 * BY * NZ + kz];
-                }
-                Dft<RY, +1>::run(cvals);
-#pragma unroll
-                for (int m = 0; m < RY; ++m) sT[m * NZ + kz] = cvals[m];
-            }
-            __syncthreads();
-            // ---- kz inverse of this warp's rows, conjugate-sensitivity coil sum ----
-            if (aL) {
-#pragma unroll
-                for (int k = 0; k < RL; ++k) u[k] = sT[m_row * NZ + jz + PZ::BFL * k];
-                Dft<RL, +1>::run(u);
-#pragma unroll
-                for (int m = 0; m < RL; ++m) sE[l * WL::EXL + jz * PZ::LS1 + m] = u[m];
-            }
-            // S rows of this coil have landed; during the first coil the x rows may stay in flight
-            if (c == 0) cp_async_wait<1>(); else cp_async_wait<0>();
-            __syncwarp();
+            for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)cur.j_y * k0) % N1);
             if (a0) {
 #pragma unroll
-                for (int k = 0; k < R0; ++k) {
-                    const cf r = sE[l * WL::EXL + k * PZ::LS1 + jz];
-                    v[k] = (k == 0) ? r : cmulc(r, twz[k]);
-                }
-                Dft<R0, +1>::run(v);
-#pragma unroll
-                for (int m = 0; m < R0; ++m) {
-                    const cf sv = cS[jz + PZ::BF0 * m];
-                    acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
-                    acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
-                }
+                for (int m = 0; m < R0; ++m) xreg[m] = a.x[cur.x_off + jz + PZ::BF0 * m];
             }
-            __syncwarp();                                    // S rows consumed: fetch the coming coil's
-            if (c + 1 < a.C) issue_s(cur, c + 1);
-            else if (has_next) issue_s(nx, 0);
-            __syncthreads();          // tile and exchange area are reused by the next coil
+#pragma unroll
+            for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
         }
-        // ---- update: the x rows are complete once everything but the newest group has landed ----
-        if (has_next) cp_async_wait<1>(); else cp_async_wait<0>();
+        const cf* cV = sV + (step & 1) * RI::TILE_V;
+        const cf* cS = sS + (step & 1) * WL::TILE + l * NZ;
+        cf v[R0], u[RL];
+        // ---- inverse radix-RY across the rows, one kz column per thread ----
+        for (int kz = threadIdx.x; kz < NZ; kz += RT::THREADS) {
+            cf cvals[RY];
+#pragma unroll
+            for (int k0 = 0; k0 < RY; ++k0) {
+                const cf r = cV[k0 * NZ + kz];
+                cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
+            }
+            Dft<RY, +1>::run(cvals);
+#pragma unroll
+            for (int m = 0; m < RY; ++m) sT[m * NZ + kz] = cvals[m];
+        }
+        __syncthreads();                                     // tile complete, column buffer free
+        issue_v(step + 2);
+        // ---- kz inverse of this warp's rows, conjugate-sensitivity coil sum ----
+        if (aL) {
+#pragma unroll
+            for (int k = 0; k < RL; ++k) u[k] = sT[m_row * NZ + jz + PZ::BFL * k];
+            Dft<RL, +1>::run(u);
+#pragma unroll
+            for (int m = 0; m < RL; ++m) sE[l * WL::EXL + jz * PZ::LS1 + m] = u[m];
+        }
+        cp_async_wait<3>();                                  // S(step); newer: V(step+1) S(step+1) V(step+2)
         __syncwarp();
         if (a0) {
 #pragma unroll
+            for (int k = 0; k < R0; ++k) {
+                const cf r = sE[l * WL::EXL + k * PZ::LS1 + jz];
+                v[k] = (k == 0) ? r : cmulc(r, twz[k]);
+            }
+            Dft<R0, +1>::run(v);
+#pragma unroll
             for (int m = 0; m < R0; ++m) {
-                const cf xv = sX[l * NZ + jz + PZ::BF0 * m];
-                a.out[cur.x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
+                const cf sv = cS[jz + PZ::BF0 * m];
+                acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
+                acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
             }
         }
-        __syncwarp();                                        // x rows read: the next item may overwrite them
-        if (!has_next) break;
-        item = nxt;
-        cur = nx;
+        __syncwarp();                                        // S rows consumed: the buffer takes step + 2
+        issue_s(step + 2);
+        if (c + 1 == C && a0) {                              // last coil of the item: the update
+#pragma unroll
+            for (int m = 0; m < R0; ++m)
+                a.out[cur.x_off + jz + PZ::BF0 * m] =
+                    make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y));
+        }
+        cp_async_wait<3>();                                  // V(step+1); newer: S(step+1) V(step+2) S(step+2)
+        __syncthreads();          // tile and exchange area are reused; next columns visible to all
     }
+    cp_async_wait<0>();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -503,7 +503,7 @@ struct PairImpl {
         if (e != cudaSuccess) return e;
         const long long items = images * a.G * BY;
         if (items <= 0) return cudaSuccess;
-        if (items > 2147483647LL) return cudaErrorInvalidConfiguration;
+        if (items * a.C > 2147483647LL) return cudaErrorInvalidConfiguration;
         static int sms = 0;                                   // one persistent block per SM
         if (sms == 0) {
             int dev = 0;

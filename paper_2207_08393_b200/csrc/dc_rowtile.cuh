@@ -216,175 +216,6 @@ rowtile_kernel(const TileArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// pass 3, persistent form: one block per SM walks over its (b,t,slab,j) items and their coils as
-// one flat sequence of steps s = (item, coil) and keeps the loads of two steps in flight: the
-// workspace columns V(s) and the sensitivity rows S(s) arrive by cp.async in double-buffered
-// shared memory, and the copies for step s+2 are issued as soon as step s has consumed its
-// buffer, across item boundaries.  At one block per SM (the coil sum, x and both twiddle sets live
-// in registers) one step of loads in flight does not cover the memory latency.
-// Commit groups are issued in the fixed order V(0) S(0) V(1) S(1) | V(s+2) S(s+2) per step, empty
-// where the sequence has ended, so that "all but the newest three" is always the wait that a
-// consumer needs.
-// ---------------------------------------------------------------------------------------------
-template <class PZ, int RY, int BY>
-struct RowTileInv {
-    using RT = RowTile<PZ, RY, BY>;
-    using WL = typename RT::WL;
-    static constexpr int TILE_V = RY * PZ::N;                            // one workspace column set
-    static constexpr int PER_WARP = RT::PER_WARP + WL::TILE;             // second buffer of S rows
-    static constexpr int OFF_V = RT::TILE_T;
-    static constexpr int OFF_WARP = RT::TILE_T + 2 * TILE_V;
-    static constexpr size_t SMEM_BYTES = sizeof(cf) * (OFF_WARP + RT::WARPS * PER_WARP + 2);
-};
-
-template <class PZ, int RY, int BY>
-__global__ void __launch_bounds__(RowTile<PZ, RY, BY>::THREADS, 1)
-rowtile_inv_kernel(const TileArgs a, const unsigned nitems) {
-    using RT = RowTile<PZ, RY, BY>;
-    using RI = RowTileInv<PZ, RY, BY>;
-    using WL = typename RT::WL;
-    constexpr int NZ = PZ::N, R0 = PZ::R0, RL = PZ::RL, TPL = WL::TPL, LW = WL::LW, N1 = RY * BY;
-    extern __shared__ __align__(16) float2 smem[];
-    cf* sT = smem;
-    cf* sV = smem + RI::OFF_V;                               // [2][RY][NZ]
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    cf* wsm = smem + RI::OFF_WARP + warp * RI::PER_WARP;
-    cf* sS = wsm;                                            // [2][LW][NZ]
-    cf* sE = wsm + 2 * WL::TILE;
-
-    const int l = lane / TPL, jz = lane % TPL;
-    const int m_row = warp * LW + l;                         // 0 .. RY-1
-    const bool a0 = jz < PZ::BF0, aL = jz < PZ::BFL;
-    const long long V3 = (long long)a.n0 * N1 * NZ;
-    const long long s_stride = (long long)a.Ts * V3;
-    const unsigned C = (unsigned)a.C;
-    if (blockIdx.x >= nitems) return;
-    const unsigned my_items = (nitems - blockIdx.x + gridDim.x - 1) / gridDim.x;
-    const unsigned total = my_items * C;                     // steps of this block (host: items * C < 2^32)
-
-    struct Item { unsigned j_y, gi; int b, t; long long x_off, s_off; };
-    auto decode = [&](unsigned step) -> Item {               // item of step s = (s / C)-th item of this block
-        const unsigned item = blockIdx.x + (step / C) * gridDim.x;
-        Item it;
-        it.j_y = item % BY;
-        it.gi = (item / BY) % (unsigned)a.G;
-        const unsigned bt = item / (BY * (unsigned)a.G);
-        it.b = (int)(bt / (unsigned)a.T);
-        it.t = (int)(bt - (unsigned)it.b * a.T);
-        const int ky = (int)it.j_y + BY * m_row;             // image-side row of this lane
-        const long long row_elems = ((long long)(a.i0_start + (int)it.gi) * N1 + ky) * NZ;
-        it.x_off = (long long)bt * V3 + row_elems;
-        it.s_off = ((long long)(it.b * a.C) * a.Ts + (a.Ts > 1 ? it.t : 0)) * V3 + row_elems;
-        return it;
-    };
-    // workspace columns of step s -> sV[s & 1]: V[unit][gi][k0][j][kz], all RY rows k0 (one commit group)
-    auto issue_v = [&](unsigned step) {
-        if (step < total) {
-            const Item it = decode(step);
-            const long long unit = ((long long)(it.b * a.C + (int)(step % C))) * a.T + it.t;
-            const cf* src = a.V + (((unit * a.G + it.gi) * RY) * (long long)BY + it.j_y) * NZ;
-            cf* dst = sV + (step & 1) * RI::TILE_V;
-            for (int i = threadIdx.x; i < RY * (NZ / 2); i += RT::THREADS) {
-                const int k0 = i / (NZ / 2), part = i - k0 * (NZ / 2);
-                cp_async16(dst + k0 * NZ + 2 * part, src + (long long)k0 * BY * NZ + 2 * part);
-            }
-        }
-        cp_async_commit();
-    };
-    // sensitivity rows of this warp for step s -> sS[s & 1] (one commit group)
-    auto issue_s = [&](unsigned step) {
-        if (step < total) {
-            const Item it = decode(step);
-            cf* dst = sS + (step & 1) * WL::TILE;
-#pragma unroll
-            for (int ll = 0; ll < LW; ++ll) {
-                const long long so = __shfl_sync(0xffffffffu, it.s_off, ll * TPL);
-                const cf* src = a.sens + so + (long long)(step % C) * s_stride;
-                for (int i = lane; i < NZ / 2; i += 32) cp_async16(dst + ll * NZ + 2 * i, src + 2 * i);
-            }
-        }
-        cp_async_commit();
-    };
-
-    cf twz[R0];                                              // kz inter-stage twiddles of this lane
-#pragma unroll
-    for (int k = 0; k < R0; ++k) twz[k] = unit_root_fwd<NZ>((jz * k) % NZ);
-
-    issue_v(0); issue_s(0); issue_v(1); issue_s(1);
-    cp_async_wait<3>();                                      // V(0)
-    __syncthreads();
-
-    Item cur = decode(0);
-    cf twy[RY], xreg[R0], acc[R0];
-    for (unsigned step = 0; step < total; ++step) {
-        const unsigned c = step % C;
-        if (c == 0) {                                        // a new item: its rows of x, its ky twiddles
-            cur = decode(step);
-#pragma unroll
-            for (int k0 = 0; k0 < RY; ++k0) twy[k0] = unit_root_fwd<N1>(((int)cur.j_y * k0) % N1);
-            if (a0) {
-#pragma unroll
-                for (int m = 0; m < R0; ++m) xreg[m] = a.x[cur.x_off + jz + PZ::BF0 * m];
-            }
-#pragma unroll
-            for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
-        }
-        const cf* cV = sV + (step & 1) * RI::TILE_V;
-        const cf* cS = sS + (step & 1) * WL::TILE + l * NZ;
-        cf v[R0], u[RL];
-        // ---- inverse radix-RY across the rows, one kz column per thread ----
-        for (int kz = threadIdx.x; kz < NZ; kz += RT::THREADS) {
-            cf cvals[RY];
-#pragma unroll
-            for (int k0 = 0; k0 < RY; ++k0) {
-                const cf r = cV[k0 * NZ + kz];
-                cvals[k0] = (k0 == 0) ? r : cmulc(r, twy[k0]);
-            }
-            Dft<RY, +1>::run(cvals);
-#pragma unroll
-            for (int m = 0; m < RY; ++m) sT[m * NZ + kz] = cvals[m];
-        }
-        __syncthreads();                                     // tile complete, column buffer free
-        issue_v(step + 2);
-        // ---- kz inverse of this warp's rows, conjugate-sensitivity coil sum ----
-        if (aL) {
-#pragma unroll
-            for (int k = 0; k < RL; ++k) u[k] = sT[m_row * NZ + jz + PZ::BFL * k];
-            Dft<RL, +1>::run(u);
-#pragma unroll
-            for (int m = 0; m < RL; ++m) sE[l * WL::EXL + jz * PZ::LS1 + m] = u[m];
-        }
-        cp_async_wait<3>();                                  // S(step); newer: V(step+1) S(step+1) V(step+2)
-        __syncwarp();
-        if (a0) {
-#pragma unroll
-            for (int k = 0; k < R0; ++k) {
-                const cf r = sE[l * WL::EXL + k * PZ::LS1 + jz];
-                v[k] = (k == 0) ? r : cmulc(r, twz[k]);
-            }
-            Dft<R0, +1>::run(v);
-#pragma unroll
-            for (int m = 0; m < R0; ++m) {
-                const cf sv = cS[jz + PZ::BF0 * m];
-                acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
-                acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
-            }
-        }
-        __syncwarp();                                        // S rows consumed: the buffer takes step + 2
-        issue_s(step + 2);
-        if (c + 1 == C && a0) {                              // last coil of the item: the update
-#pragma unroll
-            for (int m = 0; m < R0; ++m)
-                a.out[cur.x_off + jz + PZ::BF0 * m] =
-                    make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y));
-        }
-        cp_async_wait<3>();                                  // V(step+1); newer: S(step+1) V(step+2) S(step+2)
-        __syncthreads();          // tile and exchange area are reused; next columns visible to all
-    }
-    cp_async_wait<0>();
-}
-
-// ---------------------------------------------------------------------------------------------
 // pass 2: radix-BY transform over j, mask and z, inverse; one kz column per thread, no shared memory
 // ---------------------------------------------------------------------------------------------
 template <int NZ, int RY, int BY, bool HAS_Z>
@@ -496,24 +327,7 @@ struct PairImpl {
         return cudaGetLastError();
     }
     static cudaError_t fwd(const TileArgs& a, long long images, cudaStream_t s) { return rows<false>(a, images, s); }
-    static cudaError_t inv(const TileArgs& a, long long images, cudaStream_t s) {
-        using RI = RowTileInv<PZ, RY, BY>;
-        static bool done = false;
-        cudaError_t e = ensure_smem(rowtile_inv_kernel<PZ, RY, BY>, RI::SMEM_BYTES, done);
-        if (e != cudaSuccess) return e;
-        const long long items = images * a.G * BY;
-        if (items <= 0) return cudaSuccess;
-        if (items * a.C > 2147483647LL) return cudaErrorInvalidConfiguration;
-        static int sms = 0;                                   // one persistent block per SM
-        if (sms == 0) {
-            int dev = 0;
-            if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-            if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        }
-        const unsigned grid = (unsigned)(items < sms ? items : sms);
-        rowtile_inv_kernel<PZ, RY, BY><<<grid, RT::THREADS, RI::SMEM_BYTES, s>>>(a, (unsigned)items);
-        return cudaGetLastError();
-    }
+    static cudaError_t inv(const TileArgs& a, long long images, cudaStream_t s) { return rows<true>(a, images, s); }
     static cudaError_t mid(const TileArgs& a, cudaStream_t s) {
         constexpr int NZ = PZ::N;
         const int threads = NZ < 256 ? ((NZ + 31) / 32) * 32 : 256;

@@ -157,6 +157,22 @@ GLEAM_API int gleam_dc_forward_static(const void* x, const void* y, const void* 
                                       void* out, const gleam_dims* dims);
 GLEAM_API uint64_t gleam_dc_static_scratch_bytes(void);
 
+/* ---- unrolled iterations with the same measurements -------------------------------------------
+ * Every unrolled iteration (and every greedy module of Alg. 1) applies Eq. 3 with the same y and
+ * mask.  For a readout-invariant mask, what the step needs from y does not depend on x: the table
+ * z = M R^H y at the sampled phase-encode positions (R = transform along the readout axis) and the
+ * rank map of those positions.  gleam_dc_prepare computes both into dims->workspace;
+ * gleam_dc_forward_prepared then gives exactly the result of gleam_dc_forward (bit for bit) without
+ * recomputing them.  Between the two, the caller keeps that workspace untouched: no other call of
+ * this library may be given it (a gleam_dc_vjp in between needs a workspace of its own), and the
+ * mask and dims must be the same.  With GLEAM_MASK_FULL there is nothing to prepare: _prepare does
+ * nothing and _forward_prepared is gleam_dc_forward.  y is passed to both (it is read by
+ * _forward_prepared only for a full mask).  Errors as for gleam_dc_forward.
+ */
+GLEAM_API int gleam_dc_prepare(const void* y, const float* mask, const gleam_dims* dims);
+GLEAM_API int gleam_dc_forward_prepared(const void* x, const void* y, const void* sens, const float* mask,
+                                        float eta, void* out, const gleam_dims* dims);
+
 /* ---- MoDL data-consistency step (Eq. 7, second line) -------------------------------------------
  *
  *     out = (A^H A + mu I)^{-1} (A^H y + mu z)

@@ -31,7 +31,8 @@ EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam
            "gleam_status_string", "gleam_version", "gleam_dc_forward_host", "gleam_dc_vjp_host",
            "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end",
            "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes",
-           "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size"]
+           "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size",
+           "gleam_dc_prepare", "gleam_dc_forward_prepared"]
 
 KERNEL_CLASSES = ["zmap", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
                   "col_inv", "cg_vec"]
@@ -96,6 +97,10 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_dc_forward_static.restype = i32
         lib.gleam_dc_static_scratch_bytes.argtypes = []
         lib.gleam_dc_static_scratch_bytes.restype = u64
+        lib.gleam_dc_prepare.argtypes = [vp, vp, dp]
+        lib.gleam_dc_prepare.restype = i32
+        lib.gleam_dc_forward_prepared.argtypes = [vp, vp, vp, vp, f32, vp, dp]
+        lib.gleam_dc_forward_prepared.restype = i32
         lib.gleam_modl_cg_forward.argtypes = [vp, vp, vp, vp, f32, ctypes.c_int32, vp, dp]
         lib.gleam_modl_cg_forward.restype = i32
         lib.gleam_modl_cg_vjp.argtypes = [vp, vp, vp, f32, ctypes.c_int32, vp, dp]
@@ -173,6 +178,18 @@ def gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, dims: gleam_dims) -> None:
     """grad_in = grad_out - eta A^H A grad_out  (VJP of Eq. 3 with respect to x)."""
     _check(load_library().gleam_dc_vjp(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
                                         ctypes.byref(dims)))
+
+
+def gleam_dc_prepare(y, mask, dims: gleam_dims) -> None:
+    """Computes what Eq. 3 needs from y and the mask alone into dims.workspace (kept by the caller
+    until the last gleam_dc_forward_prepared)."""
+    _check(load_library().gleam_dc_prepare(_addr(y), _addr(mask), ctypes.byref(dims)))
+
+
+def gleam_dc_forward_prepared(x, y, sens, mask, eta, out, dims: gleam_dims) -> None:
+    """gleam_dc_forward with the tables of an earlier gleam_dc_prepare(y, mask, dims)."""
+    _check(load_library().gleam_dc_forward_prepared(_addr(x), _addr(y), _addr(sens), _addr(mask), float(eta),
+                                                     _addr(out), ctypes.byref(dims)))
 
 
 def gleam_dc_host_arena_size(dims: gleam_dims) -> int:
@@ -256,6 +273,17 @@ class DataConsistency:
             grad_in = self._torch.empty_like(grad_out)
         gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, self.dims())
         return grad_in
+
+    def prepare(self, y, mask):
+        """For unrolled iterations with the same y and mask: fills the workspace once; follow with
+        forward_prepared calls only (forward and vjp of this object would overwrite it)."""
+        gleam_dc_prepare(y, mask, self.dims())
+
+    def forward_prepared(self, x, y, sens, mask, eta, out=None):
+        if out is None:
+            out = self._torch.empty_like(x)
+        gleam_dc_forward_prepared(x, y, sens, mask, eta, out, self.dims())
+        return out
 
 
 def gleam_modl_cg_workspace_size(dims: gleam_dims) -> int:

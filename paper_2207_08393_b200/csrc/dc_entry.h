@@ -5,10 +5,14 @@
 
 namespace gleam {
 
+// RUN_PREPARE: only what depends on y and the mask alone (rank map, z table) is computed and left in
+// the workspace; RUN_APPLY: the step with those tables taken from the workspace as they are.
+enum { RUN_ALL = 0, RUN_PREPARE = 1, RUN_APPLY = 2 };
+
 // out = x - eta A^H (A x - y)   (y == nullptr: out = x - eta A^H A x).  Validates its arguments,
 // enqueues on d->stream, returns GLEAM_OK or a GLEAM_ERR_* code.
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d);
+        const gleam_dims* d, int mode = RUN_ALL);
 
 // GLEAM_OK for a device (or managed) pointer, GLEAM_ERR_NOT_DEVICE_POINTER otherwise
 int check_device_ptr(const void* p);

@@ -260,9 +260,15 @@ cudaError_t prof_mark(int cls, cudaStream_t s) {
 #define LAUNCH(cls, call) do { CK(prof_mark((cls), s)); CK(call); } while (0)
 
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d) {
-    if (!d) return GLEAM_ERR_NULL_POINTER;
-    if (!x || !sens || !mask || !out) return GLEAM_ERR_NULL_POINTER;
+        const gleam_dims* d, int mode) {
+    if (!d || !mask) return GLEAM_ERR_NULL_POINTER;
+    if (mode == RUN_PREPARE) {
+        if (!y) return GLEAM_ERR_NULL_POINTER;
+        x = nullptr; sens = nullptr; out = nullptr;
+    } else if (!x || !sens || !out) {
+        return GLEAM_ERR_NULL_POINTER;
+    }
+    if (mode == RUN_APPLY && !y) return GLEAM_ERR_NULL_POINTER;
     Layout L;
     int rc = make_layout(d, y != nullptr, &L);
     if (rc != GLEAM_OK) return rc;
@@ -283,14 +289,16 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         if (rc != GLEAM_OK) return rc;
     }
     // aliasing: out may equal x exactly; nothing else may overlap an output or the workspace
-    if (out != x && overlaps(out, img_b, x, img_b)) return GLEAM_ERR_ALIAS;
-    if (overlaps(out, img_b, sens, sens_b) || overlaps(out, img_b, mask, mask_b)) return GLEAM_ERR_ALIAS;
-    if (y && overlaps(out, img_b, y, ksp_b)) return GLEAM_ERR_ALIAS;
+    if (mode != RUN_PREPARE) {
+        if (out != x && overlaps(out, img_b, x, img_b)) return GLEAM_ERR_ALIAS;
+        if (overlaps(out, img_b, sens, sens_b) || overlaps(out, img_b, mask, mask_b)) return GLEAM_ERR_ALIAS;
+        if (y && overlaps(out, img_b, y, ksp_b)) return GLEAM_ERR_ALIAS;
+    }
     if (L.total > 0) {
         const void* w = d->workspace;
-        if (overlaps(w, L.total, x, img_b) || overlaps(w, L.total, out, img_b) ||
-            overlaps(w, L.total, sens, sens_b) || overlaps(w, L.total, mask, mask_b) ||
-            (y && overlaps(w, L.total, y, ksp_b)))
+        if ((mode != RUN_PREPARE && (overlaps(w, L.total, x, img_b) || overlaps(w, L.total, out, img_b) ||
+                                     overlaps(w, L.total, sens, sens_b))) ||
+            overlaps(w, L.total, mask, mask_b) || (y && overlaps(w, L.total, y, ksp_b)))
             return GLEAM_ERR_ALIAS;
     }
 
@@ -318,16 +326,18 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             int* zstart = (int*)(ws + L.off_zstart);
             const PairOps* zpair = (L.rank == 3) ? find_pair(L.n1, L.n2) : nullptr;
             const int zry = (zpair && zpair->ry <= ZMAP_MAX_RY) ? zpair->ry : 0;
-            CK(prof_mark(GLEAM_K_PREP_M2, s));
             int* zchunk = (int*)(ws + L.off_zchunk);
             const dim3 zgrid((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images);
-            if (zgrid.x > 1) {        // a table of one chunk needs no counts of earlier chunks
-                zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 1, L.n1, L.n2, L.rank, zry);
-                CK(cudaGetLastError());
+            if (mode != RUN_APPLY) {      // RUN_APPLY: the tables of an earlier RUN_PREPARE are in the workspace
                 CK(prof_mark(GLEAM_K_PREP_M2, s));
+                if (zgrid.x > 1) {        // a table of one chunk needs no counts of earlier chunks
+                    zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 1, L.n1, L.n2, L.rank, zry);
+                    CK(cudaGetLastError());
+                    CK(prof_mark(GLEAM_K_PREP_M2, s));
+                }
+                zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 0, L.n1, L.n2, L.rank, zry);
+                CK(cudaGetLastError());
             }
-            zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 0, L.n1, L.n2, L.rank, zry);
-            CK(cudaGetLastError());
             ca.zidx = zidx; ca.zlist = zlist; ca.zcount = zcount; ca.m2c = m2c; ca.zstart = zry ? zstart : nullptr;
             ra.zidx = zidx;
             ColArgs cz = ca;
@@ -336,8 +346,9 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             const int nro = (L.rank == 2) ? L.n1 : L.n0;
             float g = gsign(nro) * gsign(L.n2) * (L.rank == 3 ? gsign(L.n1) : 1.f);
             cz.scale = g / sqrtf((float)nro * (float)pe);
-            LAUNCH(GLEAM_K_COL_Z, ((L.rank == 2) ? op1 : op0)->col(COL_Z, cz, s));
+            if (mode != RUN_APPLY) LAUNCH(GLEAM_K_COL_Z, ((L.rank == 2) ? op1 : op0)->col(COL_Z, cz, s));
         }
+        if (mode == RUN_PREPARE) { CK(prof_mark(-1, s)); return GLEAM_OK; }
         if (L.rank == 2) {
             ra.mask = mask; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
@@ -366,6 +377,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             }
         }
     } else {
+        if (mode == RUN_PREPARE) return GLEAM_OK;      // a full mask has nothing to prepare
         cf* W = (cf*)(ws + L.off_W);
         ra.W = W; ra.rpb = L.n0 * L.n1; ra.row0 = 0; ra.nrows = L.images * ra.rpb;
         LAUNCH(GLEAM_K_ROW_FWD, op2->row(ROW_FWD, ra, s));
@@ -404,6 +416,15 @@ GLEAM_API int gleam_dc_forward(const void* x, const void* y, const void* sens, c
 GLEAM_API int gleam_dc_vjp(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
                  const gleam_dims* dims) {
     return gleam::run(grad_out, nullptr, sens, mask, eta, grad_in, dims);
+}
+
+GLEAM_API int gleam_dc_prepare(const void* y, const float* mask, const gleam_dims* dims) {
+    return gleam::run(nullptr, y, nullptr, mask, 0.f, nullptr, dims, gleam::RUN_PREPARE);
+}
+
+GLEAM_API int gleam_dc_forward_prepared(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                        void* out, const gleam_dims* dims) {
+    return gleam::run(x, y, sens, mask, eta, out, dims, gleam::RUN_APPLY);
 }
 
 GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes) {

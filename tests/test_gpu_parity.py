@@ -246,3 +246,34 @@ def test_rank3_chunked_workspace_matches_whole_volume(oracle, tmp_path):
     res = np.load(tmp_path / "out.npz")
     assert int(res["ws"]) < g.gleam_dc_workspace_size(g.make_dims(1, 4, 1, 3, (12, 64, 48)))
     assert np.array_equal(res["out"], whole)
+
+
+@pytest.mark.parametrize("case", [
+    (2, 2, 3, 2, (1, 20, 46), MASK_READOUT_INVARIANT),
+    (2, 1, 4, 1, (1, 64, 320), MASK_READOUT_INVARIANT),      # three-stage plan on the contiguous axis (fallback row kernel)
+    (3, 2, 3, 1, (6, 64, 32), MASK_READOUT_INVARIANT),       # row-tile 3-D path
+    (3, 1, 2, 1, (10, 46, 32), MASK_READOUT_INVARIANT),      # general 3-D path
+    (2, 2, 3, 1, (1, 12, 16), MASK_FULL),                    # nothing to prepare
+])
+def test_prepared_forward_equals_forward(oracle, case):
+    """gleam_dc_prepare + gleam_dc_forward_prepared (unrolled iterations with the same y and mask)
+    give the bits of gleam_dc_forward, iteration after iteration, and match the oracle."""
+    import torch
+    import paper_2207_08393_b200 as g
+    rank, B, C, T, n, kind = case
+    d, x, y, sens, mask = problem(rank, B, C, T, n, kind, seed=77 + sum(n))
+    dev = torch.device("cuda:0")
+    tx, ty, ts, tm = (torch.from_numpy(a).to(dev) for a in (x, y, sens, mask))
+    dc_a = g.DataConsistency(B, C, T, rank, n, 0, kind)
+    dc_b = g.DataConsistency(B, C, T, rank, n, 0, kind)
+    dc_b.prepare(ty, tm)
+    xa, xb, xo = tx, tx, x
+    for it in range(3):
+        xa = dc_a.forward(xa, ty, ts, tm, 0.6)
+        xb = dc_b.forward_prepared(xb, ty, ts, tm, 0.6)
+        torch.cuda.synchronize()
+        assert torch.equal(xa, xb), "iteration %d differs" % it
+        xo = oracle.dc_forward(xo, y, sens, mask, 0.6, d).astype(np.complex64)
+    assert_close(xb.cpu().numpy(), xo, x, "prepared chain")
+    with pytest.raises(g.GleamError):
+        g.gleam_dc_prepare(None, tm, dc_b.dims())

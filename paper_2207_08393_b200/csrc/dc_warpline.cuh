@@ -37,7 +37,10 @@ struct WarpLine {
     // (ROW_FUSED with z; lines with more sampled positions read z straight from global memory).
     static constexpr int TILE = LW * N;
     static constexpr int KCAP = (MODE == ROW_INV) ? N : (((N + 3) / 4 + 1) / 2 * 2);
-    static constexpr int KTILE = LW * KCAP;
+    // ROW_FUSED with z: slot KCAP of every line's stage holds zero; unsampled entries point at it,
+    // which keeps the k-space update free of branches
+    static constexpr int KSTRIDE = (MODE == ROW_INV) ? KCAP : KCAP + 2;
+    static constexpr int KTILE = LW * KSTRIDE;
     static constexpr bool HAS_K = (MODE == ROW_INV) || (MODE == ROW_FUSED && HAS_Z);
     static constexpr bool HAS_X = (MODE == ROW_FUSED);   // ROW_FWD and ROW_INV keep x in registers
     static constexpr bool HAS_M = (MODE == ROW_FUSED), HAS_I = (MODE == ROW_FUSED && HAS_Z);
@@ -48,11 +51,13 @@ struct WarpLine {
     static constexpr int WARP_ELEMS_ALIGNED = (WARP_ELEMS + 1) / 2 * 2;   // keep 16-byte alignment per warp
 };
 
+template <int MODE, bool HAS_Z> __device__ __forceinline__ constexpr bool use_z_slots() { return MODE == ROW_FUSED && HAS_Z; }
+
 template <class P, int WARPS, int MODE, bool HAS_Z>
 __global__ void __launch_bounds__(WARPS * 32)
 warpline_kernel(const RowArgs a) {
     using WL = WarpLine<P, MODE, HAS_Z>;
-    constexpr int KCAP = WL::KCAP, KTILE = WL::KTILE;
+    constexpr int KCAP = WL::KCAP, KTILE = WL::KTILE, KSTRIDE = WL::KSTRIDE;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL, TPL = WL::TPL, LW = WL::LW, TILE = WL::TILE;
     extern __shared__ __align__(16) float2 smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -73,6 +78,10 @@ warpline_kernel(const RowArgs a) {
         for (int k = 0; k < R0; ++k) tw0[k] = unit_root_fwd<N>((j * k) % N);
     }
 
+    if (use_z_slots<MODE, HAS_Z>()) {
+        for (int i = lane; i < 2 * LW; i += 32) sK[(i / LW) * KTILE + (i % LW) * KSTRIDE + KCAP] = make_float2(0.f, 0.f);
+        __syncwarp();
+    }
     const long long ngroups = (a.nrows + LW - 1) / LW;
     const long long wstride = (long long)gridDim.x * WARPS;
     constexpr bool use_z = (MODE == ROW_FUSED) && HAS_Z;
@@ -109,7 +118,7 @@ warpline_kernel(const RowArgs a) {
                 for (int i = lane; i < N / 2; i += 32) cp_async16(sS + buf * TILE + ll * N + 2 * i, src + 2 * i);
                 if (use_k && kc <= KCAP) {
                     const cf* ks = ((MODE == ROW_FUSED) ? a.z : a.W) + ko + c * k_stride;
-                    for (int i = lane; i < (kc + 1) / 2; i += 32) cp_async16(sK + buf * KTILE + ll * KCAP + 2 * i, ks + 2 * i);
+                    for (int i = lane; i < (kc + 1) / 2; i += 32) cp_async16(sK + buf * KTILE + ll * KSTRIDE + 2 * i, ks + 2 * i);
                 }
             }
         };
@@ -161,7 +170,7 @@ warpline_kernel(const RowArgs a) {
             __syncwarp();
 
             const cf* cS = sS + buf * TILE + l * N;
-            const cf* cK = sK + buf * KTILE + l * KCAP;
+            const cf* cK = sK + buf * KTILE + l * KSTRIDE;
             const cf* gK = use_z ? a.z + k_off + c * k_stride : nullptr;   // this line's compact z row
             const cf* cX = sX + l * N;
             cf v[R0], u[RL];
@@ -192,15 +201,26 @@ warpline_kernel(const RowArgs a) {
             if (MODE == ROW_FUSED) {
                 if (aL) {
                     const float* mm = sM + l * N;
+                    if (use_z && row_ok && k_cnt <= KCAP) {
+                        // staged z: unsampled entries read the zero slot (lanes without a row hold no rank table)
 #pragma unroll
-                    for (int k = 0; k < RL; ++k) {
-                        const float w = mm[j + P::BFL * k];
-                        u[k] = cscale(u[k], w);
-                        if (use_z && row_ok) {      // lanes without a row hold no rank table
+                        for (int k = 0; k < RL; ++k) {
+                            const float w = mm[j + P::BFL * k];
                             const int r = sI[l * N + j + P::BFL * k];
-                            if (r >= 0 && r < N) {
-                                const cf q = (k_cnt <= KCAP) ? cK[r] : gK[r];
-                                u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
+                            const cf q = cK[(r >= 0) ? r : KCAP];
+                            u[k] = make_float2(fmaf(w, u[k].x, -q.x), fmaf(w, u[k].y, -q.y));
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < RL; ++k) {
+                            const float w = mm[j + P::BFL * k];
+                            u[k] = cscale(u[k], w);
+                            if (use_z && row_ok) {      // more sampled entries than the stage holds: from global memory
+                                const int r = sI[l * N + j + P::BFL * k];
+                                if (r >= 0 && r < N) {
+                                    const cf q = gK[r];
+                                    u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
+                                }
                             }
                         }
                     }

@@ -12,7 +12,12 @@ enum { RUN_ALL = 0, RUN_PREPARE = 1, RUN_APPLY = 2 };
 // out = x - eta A^H (A x - y)   (y == nullptr: out = x - eta A^H A x).  Validates its arguments,
 // enqueues on d->stream, returns GLEAM_OK or a GLEAM_ERR_* code.
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode = RUN_ALL);
+        const gleam_dims* d, int mode = RUN_ALL, double* dot_rows = nullptr);
+
+// dot_rows (device, one double per image row, B*T*n1): the one-pass 2-D kernel also stores
+// Re<x_row, out_row> of every row it writes, so that a caller's inner product <x, out> needs no
+// pass of its own.  Only where this returns true (2-D, readout-invariant mask, warp-resident row plan).
+bool dot_rows_supported(const gleam_dims* d);
 
 // GLEAM_OK for a device (or managed) pointer, GLEAM_ERR_NOT_DEVICE_POINTER otherwise
 int check_device_ptr(const void* p);

@@ -33,6 +33,7 @@ struct RowArgs {
     int row0;           // first row of this launch inside the full image rows
     int RPB;            // rows of a full image (n0*n1)
     long long nrows;    // B*T*rpb
+    double* dot_rows;   // ROW_FUSED (warp-resident form): if not null, Re<x, out> of every image row, (B*T*rpb)
 };
 
 struct ColArgs {

@@ -270,12 +270,19 @@ warpline_kernel(const RowArgs a) {
         }
         cp_async_wait<0>();
         if (MODE != ROW_FWD) {
+            double dsum = 0.0;       // Re<x, out> over this lane's elements (for the caller's inner product)
             if (a0 && row_ok) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
                     const cf xv = WL::HAS_X ? sX[l * N + j + P::BF0 * m] : xreg[m];
-                    a.out[x_off + j + P::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
+                    const cf ov = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
+                    a.out[x_off + j + P::BF0 * m] = ov;
+                    if (MODE == ROW_FUSED && a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;
                 }
+            }
+            if (MODE == ROW_FUSED && a.dot_rows != nullptr) {     // the same in every thread
+                for (int o = TPL / 2; o > 0; o >>= 1) dsum += __shfl_down_sync(0xffffffffu, dsum, o, TPL);
+                if (j == 0 && row_ok) a.dot_rows[row] = dsum;
             }
         }
     }

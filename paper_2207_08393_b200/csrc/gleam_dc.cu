@@ -259,8 +259,14 @@ cudaError_t prof_mark(int cls, cudaStream_t s) {
 }
 #define LAUNCH(cls, call) do { CK(prof_mark((cls), s)); CK(call); } while (0)
 
+bool dot_rows_supported(const gleam_dims* d) {
+    if (!d || d->fft_rank != 2 || d->mask_kind != GLEAM_MASK_READOUT_INVARIANT) return false;
+    const SizeOps* op2 = find_size(d->n[2]);
+    return op2 && op2->row_is_warp_resident;
+}
+
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode) {
+        const gleam_dims* d, int mode, double* dot_rows) {
     if (!d || !mask) return GLEAM_ERR_NULL_POINTER;
     if (mode == RUN_PREPARE) {
         if (!y) return GLEAM_ERR_NULL_POINTER;
@@ -269,6 +275,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         return GLEAM_ERR_NULL_POINTER;
     }
     if (mode == RUN_APPLY && !y) return GLEAM_ERR_NULL_POINTER;
+    if (dot_rows && !dot_rows_supported(d)) return GLEAM_ERR_UNIMPLEMENTED;   // callers ask first
     Layout L;
     int rc = make_layout(d, y != nullptr, &L);
     if (rc != GLEAM_OK) return rc;
@@ -351,6 +358,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         if (mode == RUN_PREPARE) { CK(prof_mark(-1, s)); return GLEAM_OK; }
         if (L.rank == 2) {
             ra.mask = mask; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
+            ra.dot_rows = dot_rows;
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
             cf* W = (cf*)(ws + L.off_W);

@@ -11,8 +11,9 @@
 //     cg_dot  : pq = Re <p,q>
 //     cg_step : alpha = rr / (mu pq);  x += alpha p;  r -= alpha mu q;  rr' = <r,r>
 //     cg_dir  : beta = rr' / rr;  p = r + beta p
-// (cg_dot, cg_step and cg_dir run as one cooperative launch with two grid-wide barriers where the
-// device allows it, as three launches otherwise)
+// Where the operator is the one-pass 2-D kernel, that kernel also stores Re<p_row, q_row> of every
+// image row it writes (it holds both in registers at its update step), cg_step adds the rows of its
+// example in index order and cg_dot is not launched.
 //
 // Inner products: every thread accumulates in double precision, blocks reduce in a fixed order and
 // store one partial sum each; the block that arrives last (a counter per example) adds the
@@ -20,11 +21,8 @@
 // result does not depend on the order in which blocks run.
 #include "dc_entry.h"
 
-#include <cooperative_groups.h>
-
 #include <cmath>
 #include <cstdint>
-#include <cstdlib>
 
 namespace gleam {
 
@@ -36,7 +34,9 @@ struct CgArgs {
     const float4* z;       // z (forward) or grad_out (VJP), two complex values per element
     const float4* q;       // A^H y at cg_init, H p / mu afterwards
     float4* r; float4* p; float4* x;
-    double* partial;       // (B, CG_MAX_BLOCKS), and a second array of the same size behind it
+    double* partial;       // (B, CG_MAX_BLOCKS)
+    const double* dot_rows;  // (B, rows_per_example): Re<p,q> per image row from the operator, or null
+    int rows_per_example;
     double* sc;            // (B, SC_STRIDE): <r,r> of even / odd steps, <p,q>
     unsigned* counter;     // (B)
     long long ne2;         // float4 elements per example
@@ -106,10 +106,28 @@ __global__ void __launch_bounds__(CG_THREADS) cg_dot_kernel(const CgArgs a) {
     reduce_to_scalar(acc, a, a.sc + (size_t)blockIdx.y * SC_STRIDE + SC_PQ);
 }
 
+template <bool FROM_ROWS>
 __global__ void __launch_bounds__(CG_THREADS) cg_step_kernel(const CgArgs a) {
     const long long base = (long long)blockIdx.y * a.ne2;
     const double* sc = a.sc + (size_t)blockIdx.y * SC_STRIDE;
-    const double rr = sc[a.parity], pq = sc[SC_PQ];
+    const double rr = sc[a.parity];
+    double pq;
+    if (FROM_ROWS) {
+        // <p,q> of this example: the operator's per-row values, added in index order (every block
+        // computes the same sum)
+        __shared__ double pq_sh;
+        if (threadIdx.x < 32) {
+            const double* rows = a.dot_rows + (size_t)blockIdx.y * a.rows_per_example;
+            double t = 0.0;
+            for (int i = threadIdx.x; i < a.rows_per_example; i += 32) t += rows[i];
+            for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
+            if (threadIdx.x == 0) pq_sh = t;
+        }
+        __syncthreads();
+        pq = pq_sh;
+    } else {
+        pq = sc[SC_PQ];
+    }
     // an example whose residual is exactly zero stays as it is
     const double alpha = (rr > 0.0 && pq > 0.0) ? rr / ((double)a.mu * pq) : 0.0;
     const float af = (float)alpha, amu = (float)(alpha * (double)a.mu);
@@ -137,104 +155,10 @@ __global__ void __launch_bounds__(CG_THREADS) cg_dir_kernel(const CgArgs a) {
     }
 }
 
-// One conjugate-gradient step after the operator call in a single cooperative launch: cg_dot,
-// cg_step and cg_dir with a grid-wide barrier where the next phase needs a finished inner product.
-// Every block adds up the partial sums of its example itself, in index order, so all blocks get the
-// same scalar.  Same arithmetic, same order of additions as the three separate kernels.
-__device__ __forceinline__ double block_partial(double v, double* warp_sum) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
-    __syncthreads();                                    // warp_sum may still be read from the last use
-    if (lane == 0) warp_sum[warp] = v;
-    __syncthreads();
-    double t = 0.0;
-    for (int w = 0; w < CG_THREADS / 32; ++w) t += warp_sum[w];
-    return t;                                           // the same value in every thread
-}
-
-__device__ __forceinline__ double sum_partials(const double* part, double* bcast) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (warp == 0) {
-        const volatile double* vp = part;
-        double t = 0.0;
-        for (unsigned i = lane; i < gridDim.x; i += 32) t += vp[i];
-        for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
-        if (lane == 0) *bcast = t;
-    }
-    __syncthreads();
-    return *bcast;
-}
-
-__global__ void __launch_bounds__(CG_THREADS) cg_fused_kernel(const CgArgs a, int with_dir) {
-    namespace cgr = cooperative_groups;
-    cgr::grid_group grid = cgr::this_grid();
-    __shared__ double warp_sum[CG_THREADS / 32];
-    __shared__ double bcast[2];
-    const long long base = (long long)blockIdx.y * a.ne2;
-    const long long first = (long long)blockIdx.x * CG_THREADS + threadIdx.x, stride = (long long)gridDim.x * CG_THREADS;
-    double* sc = a.sc + (size_t)blockIdx.y * SC_STRIDE;
-    double* partA = a.partial + (size_t)blockIdx.y * CG_MAX_BLOCKS;
-    double* partB = partA + (size_t)gridDim.y * CG_MAX_BLOCKS;
-
-    double acc = 0.0;
-    for (long long i = first; i < a.ne2; i += stride) {
-        const float4 pv = a.p[base + i], qv = a.q[base + i];
-        acc += (double)pv.x * qv.x + (double)pv.y * qv.y + (double)pv.z * qv.z + (double)pv.w * qv.w;
-    }
-    acc = block_partial(acc, warp_sum);
-    if (threadIdx.x == 0) partA[blockIdx.x] = acc;
-    __threadfence();
-    grid.sync();
-    const double pq = sum_partials(partA, &bcast[0]);
-    const double rr = sc[a.parity];
-    const double alpha = (rr > 0.0 && pq > 0.0) ? rr / ((double)a.mu * pq) : 0.0;
-    const float af = (float)alpha, amu = (float)(alpha * (double)a.mu);
-    acc = 0.0;
-    for (long long i = first; i < a.ne2; i += stride) {
-        const float4 pv = a.p[base + i], qv = a.q[base + i];
-        float4 xv = a.x[base + i], rv = a.r[base + i];
-        xv = make_float4(fmaf(af, pv.x, xv.x), fmaf(af, pv.y, xv.y), fmaf(af, pv.z, xv.z), fmaf(af, pv.w, xv.w));
-        rv = make_float4(fmaf(-amu, qv.x, rv.x), fmaf(-amu, qv.y, rv.y), fmaf(-amu, qv.z, rv.z), fmaf(-amu, qv.w, rv.w));
-        a.x[base + i] = xv;
-        a.r[base + i] = rv;
-        acc += norm2(rv);
-    }
-    acc = block_partial(acc, warp_sum);
-    if (threadIdx.x == 0) partB[blockIdx.x] = acc;
-    __threadfence();
-    grid.sync();
-    const double rr_new = sum_partials(partB, &bcast[1]);
-    if (blockIdx.x == 0 && threadIdx.x == 0) { sc[a.parity ^ 1] = rr_new; sc[SC_PQ] = pq; }
-    if (!with_dir) return;
-    const float beta = (rr > 0.0) ? (float)(rr_new / rr) : 0.f;
-    for (long long i = first; i < a.ne2; i += stride) {
-        const float4 rv = a.r[base + i], pv = a.p[base + i];
-        a.p[base + i] = make_float4(fmaf(beta, pv.x, rv.x), fmaf(beta, pv.y, rv.y), fmaf(beta, pv.z, rv.z), fmaf(beta, pv.w, rv.w));
-    }
-}
-
-// Blocks of cg_fused_kernel that can be resident at once on the current device (0: cooperative
-// launches are not available, or switched off with GLEAM_CG_FUSED=0; read once per process).
-static int fused_capacity() {
-    static int cap = -1;
-    if (cap < 0) {
-        cap = 0;
-        const char* e = getenv("GLEAM_CG_FUSED");
-        int dev = 0, coop = 0, sms = 0, per_sm = 0;
-        if (!(e && e[0] == '0') && cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop &&
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cg_fused_kernel, CG_THREADS, 0) == cudaSuccess)
-            cap = sms * per_sm;
-        cudaGetLastError();
-    }
-    return cap;
-}
-
 static inline uint64_t up256(uint64_t v) { return (v + 255) / 256 * 256; }
 
 struct CgLayout {
-    uint64_t dc_bytes, img_bytes, off_q, off_r, off_p, off_partial, off_sc, off_counter, total;
+    uint64_t dc_bytes, img_bytes, off_q, off_r, off_p, off_partial, off_rows, off_sc, off_counter, total;
     long long ne2;
     int B;
 };
@@ -254,7 +178,8 @@ static int cg_layout(const gleam_dims* d, CgLayout* L) {
     L->off_q = off; off = up256(off + L->img_bytes);
     L->off_r = off; off = up256(off + L->img_bytes);
     L->off_p = off; off = up256(off + L->img_bytes);
-    L->off_partial = off; off = up256(off + 2u * (uint64_t)d->batch * CG_MAX_BLOCKS * sizeof(double));
+    L->off_partial = off; off = up256(off + (uint64_t)d->batch * CG_MAX_BLOCKS * sizeof(double));
+    L->off_rows = off; off = up256(off + (uint64_t)d->batch * d->frames * d->n[1] * sizeof(double));
     L->off_sc = off; off = up256(off + (uint64_t)d->batch * SC_STRIDE * sizeof(double));
     L->off_counter = off; off = up256(off + (uint64_t)d->batch * sizeof(unsigned));
     L->total = off;
@@ -311,12 +236,10 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
     if (nb < 1) nb = 1;
     if (nb > CG_MAX_BLOCKS) nb = CG_MAX_BLOCKS;
     const dim3 grid((unsigned)nb, (unsigned)L.B);
-    // the fused step needs all its blocks resident at once: fewer blocks per example if need be
-    const int cap = fused_capacity();
-    const bool fused = cap >= L.B;
-    long long nbf = nb;
-    if (fused && nbf * L.B > cap) nbf = cap / L.B;
-    const dim3 grid_fused((unsigned)nbf, (unsigned)L.B);
+    // the one-pass 2-D operator kernel delivers <p,q> per image row
+    const bool from_rows = dot_rows_supported(d);
+    double* dot_rows = from_rows ? (double*)(ws + L.off_rows) : nullptr;
+    a.dot_rows = dot_rows; a.rows_per_example = d->frames * d->n[1];
 
     CGCK(cudaMemsetAsync(ws + L.off_sc, 0, L.total - L.off_sc, s));          // scalars and counters
     if (y) {
@@ -332,20 +255,19 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
     CGCK(cudaGetLastError());
     for (int k = 0; k < n_iter; ++k) {
         a.parity = k & 1;
-        CGRUN(run(a.p, nullptr, sens, mask, -1.0f / mu, ws + L.off_q, &dd));     // q = H p / mu
-        if (fused) {
-            int with_dir = (k + 1 < n_iter) ? 1 : 0;
-            void* kargs[2] = {(void*)&a, (void*)&with_dir};
+        CGRUN(run(a.p, nullptr, sens, mask, -1.0f / mu, ws + L.off_q, &dd, RUN_ALL, dot_rows));     // q = H p / mu
+        if (from_rows) {
             CGCK(prof_mark(GLEAM_K_CG_VEC, s));
-            CGCK(cudaLaunchCooperativeKernel((const void*)cg_fused_kernel, grid_fused, dim3(CG_THREADS), kargs, 0, s));
-            continue;
+            cg_step_kernel<true><<<grid, CG_THREADS, 0, s>>>(a);
+            CGCK(cudaGetLastError());
+        } else {
+            CGCK(prof_mark(GLEAM_K_CG_VEC, s));
+            cg_dot_kernel<<<grid, CG_THREADS, 0, s>>>(a);
+            CGCK(cudaGetLastError());
+            CGCK(prof_mark(GLEAM_K_CG_VEC, s));
+            cg_step_kernel<false><<<grid, CG_THREADS, 0, s>>>(a);
+            CGCK(cudaGetLastError());
         }
-        CGCK(prof_mark(GLEAM_K_CG_VEC, s));
-        cg_dot_kernel<<<grid, CG_THREADS, 0, s>>>(a);
-        CGCK(cudaGetLastError());
-        CGCK(prof_mark(GLEAM_K_CG_VEC, s));
-        cg_step_kernel<<<grid, CG_THREADS, 0, s>>>(a);
-        CGCK(cudaGetLastError());
         if (k + 1 < n_iter) {
             CGCK(prof_mark(GLEAM_K_CG_VEC, s));
             cg_dir_kernel<<<grid, CG_THREADS, 0, s>>>(a);

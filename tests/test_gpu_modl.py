@@ -71,6 +71,8 @@ def test_rank2_steps_and_mu(oracle, n_iter, mu):
     (3, 1, 2, 2, (4, 6, 8), MASK_FULL, 1, False),
     (3, 2, 3, 1, (10, 46, 32), MASK_READOUT_INVARIANT, 0, True),
     (2, 1, 2, 1, (1, 2, 2), MASK_READOUT_INVARIANT, 0, False),       # smallest supported image
+    (2, 2, 3, 2, (1, 16, 320), MASK_READOUT_INVARIANT, 0, False),    # three-stage row plan: <p,q> by its own kernel
+    (2, 3, 2, 1, (1, 10, 160), MASK_READOUT_INVARIANT, 0, True),     # <p,q> per row from the operator, ragged line groups
 ])
 def test_shapes_and_masks(oracle, case):
     rank, B, C, T, n, kind, shf, weighted = case
@@ -161,29 +163,3 @@ def test_error_codes():
     g.gleam_modl_cg_forward(z, y, s, m, 0.05, 10, z, d)          # exact alias is allowed
     torch.cuda.synchronize()
 
-
-def test_three_launch_step_matches_fused_step(oracle, tmp_path):
-    """The conjugate-gradient step runs as one cooperative launch where the device allows it and as
-    three launches otherwise (GLEAM_CG_FUSED=0 selects the latter, read once per process): a child
-    process on the three-launch path must match the oracle and agree with the fused path to
-    rounding of the inner products."""
-    import os
-    import subprocess
-    import sys
-    d, z, y, sens, mask = problem(2, 2, 4, 2, (1, 48, 40), MASK_READOUT_INVARIANT, seed=31)
-    fused = run_gpu_modl(z, y, sens, mask, 0.05, 10, 2, 0, MASK_READOUT_INVARIANT)
-    ref = oracle.modl_cg_forward(z, y, sens, mask, 0.05, 10, d)
-    close(fused, ref, "fused")
-    np.savez(tmp_path / "in.npz", z=z, y=y, sens=sens, mask=mask)
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    code = (
-        "import sys, numpy as np; sys.path.insert(0, %r)\n"
-        "from tests.gpu_common import run_gpu_modl\n"
-        "z = np.load(%r)\n"
-        "out = run_gpu_modl(z['z'], z['y'], z['sens'], z['mask'], 0.05, 10, 2, 0, 1)\n"
-        "np.savez(%r, out=out)\n"
-    ) % (root, str(tmp_path / "in.npz"), str(tmp_path / "out.npz"))
-    subprocess.run([sys.executable, "-c", code], check=True, env=dict(os.environ, GLEAM_CG_FUSED="0"), timeout=600)
-    three = np.load(tmp_path / "out.npz")["out"]
-    close(three, ref, "three launches")
-    assert np.abs(three - fused).max() <= 1e-5 * np.abs(ref).max()

@@ -7,18 +7,20 @@
 // operator kernel changes.  The right-hand side A^H y is the forward call on a zero image with
 // eta = 1.  What remains are image-sized vector updates with inner products per batch example:
 //
-//     cg_init : b = A^H y + mu z  (VJP: b = mu g);  r = p = b;  x = 0;  rr = <b,b>
-//     cg_dot  : pq = Re <p,q>
-//     cg_step : alpha = rr / (mu pq);  x += alpha p;  r -= alpha mu q;  rr' = <r,r>
+//     cg_init : b = A^H y + mu z  (VJP: b = mu g);  r = p = b;  x = 0;  partial sums of <b,b>
+//     cg_dot  : partial sums of Re <p,q>
+//     cg_step : alpha = rr / (mu pq);  x += alpha p;  r -= alpha mu q;  partial sums of <r,r>
 //     cg_dir  : beta = rr' / rr;  p = r + beta p
-// Where the operator is the one-pass 2-D kernel, that kernel also stores Re<p_row, q_row> of every
-// image row it writes (it holds both in registers at its update step), cg_step adds the rows of its
-// example in index order and cg_dot is not launched.
 //
-// Inner products: every thread accumulates in double precision, blocks reduce in a fixed order and
-// store one partial sum each; the block that arrives last (a counter per example) adds the
-// partial sums in index order and stores the scalar.  No block waits for another one, and the
-// result does not depend on the order in which blocks run.
+// Where the operator is the one-pass 2-D kernel, that kernel also stores Re<p_row, q_row> of every
+// image row it writes (it holds both in registers at its update step) and cg_dot is not launched.
+//
+// Inner products: every thread accumulates in double precision, a block reduces in a fixed order
+// and stores one partial sum; the kernel that needs the scalar adds the partial sums of its example
+// in a fixed order at its start (every block the same sum).  Producer and consumer are different
+// launches on one stream: no atomics, no fences, no block waits for another one, and the result
+// does not depend on the order in which blocks run.  <r,r> alternates between two partial-sum
+// arrays (step parity) because cg_dir needs the old and the new value.
 #include "dc_entry.h"
 
 #include <cmath>
@@ -28,49 +30,42 @@ namespace gleam {
 
 constexpr int CG_THREADS = 256;
 constexpr int CG_MAX_BLOCKS = 592;          // partial sums per example (4 blocks per SM on 148 SMs)
-enum { SC_RR0 = 0, SC_RR1 = 1, SC_PQ = 2, SC_STRIDE = 4 };
 
 struct CgArgs {
-    const float4* z;       // z (forward) or grad_out (VJP), two complex values per element
-    const float4* q;       // A^H y at cg_init, H p / mu afterwards
+    const float4* z;         // z (forward) or grad_out (VJP), two complex values per element
+    const float4* q;         // A^H y at cg_init, H p / mu afterwards
     float4* r; float4* p; float4* x;
-    double* partial;       // (B, CG_MAX_BLOCKS)
+    double* part_rr;         // (2, B, CG_MAX_BLOCKS): <r,r> partial sums of even / odd steps
+    double* part_pq;         // (B, CG_MAX_BLOCKS): <p,q> partial sums written by cg_dot
     const double* dot_rows;  // (B, rows_per_example): Re<p,q> per image row from the operator, or null
     int rows_per_example;
-    double* sc;            // (B, SC_STRIDE): <r,r> of even / odd steps, <p,q>
-    unsigned* counter;     // (B)
-    long long ne2;         // float4 elements per example
+    long long ne2;           // float4 elements per example
     float mu;
-    int parity;            // step k & 1: sc[parity] holds <r_k, r_k>
+    int parity;              // step k & 1: part_rr[parity] holds <r_k, r_k>
 };
 
-// Sum of v over the block in a fixed order, then over the blocks of this example through the
-// partial-sum array; the last block to arrive stores the total in *dst.
-__device__ __forceinline__ void reduce_to_scalar(double v, const CgArgs& a, double* dst) {
+// Sum of v over the block in a fixed order; the same value in every thread.
+__device__ __forceinline__ double block_sum(double v) {
     __shared__ double warp_sum[CG_THREADS / 32];
-    __shared__ bool is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    __syncthreads();                                    // earlier readers of warp_sum are done
     if (lane == 0) warp_sum[warp] = v;
     __syncthreads();
-    const unsigned b = blockIdx.y;
-    if (threadIdx.x == 0) {
-        double t = 0.0;
-        for (int w = 0; w < CG_THREADS / 32; ++w) t += warp_sum[w];
-        a.partial[(size_t)b * CG_MAX_BLOCKS + blockIdx.x] = t;
-        __threadfence();
-        const unsigned ticket = atomicAdd(&a.counter[b], 1u);
-        is_last = (ticket == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (is_last && warp == 0) {
-        __threadfence();
-        const volatile double* part = a.partial + (size_t)b * CG_MAX_BLOCKS;
-        double t = 0.0;
-        for (unsigned i = lane; i < gridDim.x; i += 32) t += part[i];
-        for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
-        if (lane == 0) { *dst = t; a.counter[b] = 0u; }
-    }
+    double t = 0.0;
+    for (int w = 0; w < CG_THREADS / 32; ++w) t += warp_sum[w];
+    return t;
+}
+
+// Sum of n values written by an earlier launch (fixed order: thread t takes t, t + 256, ...).
+__device__ __forceinline__ double array_sum(const double* v, int n) {
+    double t = 0.0;
+    for (int i = threadIdx.x; i < n; i += CG_THREADS) t += __ldcg(v + i);
+    return block_sum(t);
+}
+
+__device__ __forceinline__ double* rr_slot(const CgArgs& a, int which) {
+    return a.part_rr + ((size_t)which * gridDim.y + blockIdx.y) * CG_MAX_BLOCKS;
 }
 
 __device__ __forceinline__ double norm2(float4 v) {
@@ -93,7 +88,8 @@ __global__ void __launch_bounds__(CG_THREADS) cg_init_kernel(const CgArgs a) {
         a.x[base + i] = make_float4(0.f, 0.f, 0.f, 0.f);
         acc += norm2(b);
     }
-    reduce_to_scalar(acc, a, a.sc + (size_t)blockIdx.y * SC_STRIDE + SC_RR0);
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) rr_slot(a, 0)[blockIdx.x] = acc;
 }
 
 __global__ void __launch_bounds__(CG_THREADS) cg_dot_kernel(const CgArgs a) {
@@ -103,31 +99,16 @@ __global__ void __launch_bounds__(CG_THREADS) cg_dot_kernel(const CgArgs a) {
         const float4 pv = a.p[base + i], qv = a.q[base + i];
         acc += (double)pv.x * qv.x + (double)pv.y * qv.y + (double)pv.z * qv.z + (double)pv.w * qv.w;
     }
-    reduce_to_scalar(acc, a, a.sc + (size_t)blockIdx.y * SC_STRIDE + SC_PQ);
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) a.part_pq[(size_t)blockIdx.y * CG_MAX_BLOCKS + blockIdx.x] = acc;
 }
 
 template <bool FROM_ROWS>
 __global__ void __launch_bounds__(CG_THREADS) cg_step_kernel(const CgArgs a) {
     const long long base = (long long)blockIdx.y * a.ne2;
-    const double* sc = a.sc + (size_t)blockIdx.y * SC_STRIDE;
-    const double rr = sc[a.parity];
-    double pq;
-    if (FROM_ROWS) {
-        // <p,q> of this example: the operator's per-row values, added in index order (every block
-        // computes the same sum)
-        __shared__ double pq_sh;
-        if (threadIdx.x < 32) {
-            const double* rows = a.dot_rows + (size_t)blockIdx.y * a.rows_per_example;
-            double t = 0.0;
-            for (int i = threadIdx.x; i < a.rows_per_example; i += 32) t += rows[i];
-            for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xffffffffu, t, o);
-            if (threadIdx.x == 0) pq_sh = t;
-        }
-        __syncthreads();
-        pq = pq_sh;
-    } else {
-        pq = sc[SC_PQ];
-    }
+    const double rr = array_sum(rr_slot(a, a.parity), (int)gridDim.x);
+    const double pq = FROM_ROWS ? array_sum(a.dot_rows + (size_t)blockIdx.y * a.rows_per_example, a.rows_per_example)
+                                : array_sum(a.part_pq + (size_t)blockIdx.y * CG_MAX_BLOCKS, (int)gridDim.x);
     // an example whose residual is exactly zero stays as it is
     const double alpha = (rr > 0.0 && pq > 0.0) ? rr / ((double)a.mu * pq) : 0.0;
     const float af = (float)alpha, amu = (float)(alpha * (double)a.mu);
@@ -141,13 +122,14 @@ __global__ void __launch_bounds__(CG_THREADS) cg_step_kernel(const CgArgs a) {
         a.r[base + i] = rv;
         acc += norm2(rv);
     }
-    reduce_to_scalar(acc, a, a.sc + (size_t)blockIdx.y * SC_STRIDE + (a.parity ^ 1));
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) rr_slot(a, a.parity ^ 1)[blockIdx.x] = acc;
 }
 
 __global__ void __launch_bounds__(CG_THREADS) cg_dir_kernel(const CgArgs a) {
     const long long base = (long long)blockIdx.y * a.ne2;
-    const double* sc = a.sc + (size_t)blockIdx.y * SC_STRIDE;
-    const double rr = sc[a.parity], rr_new = sc[a.parity ^ 1];
+    const double rr = array_sum(rr_slot(a, a.parity), (int)gridDim.x);
+    const double rr_new = array_sum(rr_slot(a, a.parity ^ 1), (int)gridDim.x);
     const float beta = (rr > 0.0) ? (float)(rr_new / rr) : 0.f;
     for (long long i = (long long)blockIdx.x * CG_THREADS + threadIdx.x; i < a.ne2; i += (long long)gridDim.x * CG_THREADS) {
         const float4 rv = a.r[base + i], pv = a.p[base + i];
@@ -158,7 +140,7 @@ __global__ void __launch_bounds__(CG_THREADS) cg_dir_kernel(const CgArgs a) {
 static inline uint64_t up256(uint64_t v) { return (v + 255) / 256 * 256; }
 
 struct CgLayout {
-    uint64_t dc_bytes, img_bytes, off_q, off_r, off_p, off_partial, off_rows, off_sc, off_counter, total;
+    uint64_t dc_bytes, img_bytes, off_q, off_r, off_p, off_rr, off_pq, off_rows, total;
     long long ne2;
     int B;
 };
@@ -178,10 +160,9 @@ static int cg_layout(const gleam_dims* d, CgLayout* L) {
     L->off_q = off; off = up256(off + L->img_bytes);
     L->off_r = off; off = up256(off + L->img_bytes);
     L->off_p = off; off = up256(off + L->img_bytes);
-    L->off_partial = off; off = up256(off + (uint64_t)d->batch * CG_MAX_BLOCKS * sizeof(double));
+    L->off_rr = off; off = up256(off + 2u * (uint64_t)d->batch * CG_MAX_BLOCKS * sizeof(double));
+    L->off_pq = off; off = up256(off + (uint64_t)d->batch * CG_MAX_BLOCKS * sizeof(double));
     L->off_rows = off; off = up256(off + (uint64_t)d->batch * d->frames * d->n[1] * sizeof(double));
-    L->off_sc = off; off = up256(off + (uint64_t)d->batch * SC_STRIDE * sizeof(double));
-    L->off_counter = off; off = up256(off + (uint64_t)d->batch * sizeof(unsigned));
     L->total = off;
     return GLEAM_OK;
 }
@@ -230,7 +211,7 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
     CgArgs a{};
     a.z = (const float4*)z; a.q = (const float4*)(ws + L.off_q);
     a.r = (float4*)(ws + L.off_r); a.p = (float4*)(ws + L.off_p); a.x = (float4*)out;
-    a.partial = (double*)(ws + L.off_partial); a.sc = (double*)(ws + L.off_sc); a.counter = (unsigned*)(ws + L.off_counter);
+    a.part_rr = (double*)(ws + L.off_rr); a.part_pq = (double*)(ws + L.off_pq);
     a.ne2 = L.ne2; a.mu = mu; a.parity = 0;
     long long nb = (L.ne2 + (long long)CG_THREADS * 4 - 1) / ((long long)CG_THREADS * 4);
     if (nb < 1) nb = 1;
@@ -241,7 +222,6 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
     double* dot_rows = from_rows ? (double*)(ws + L.off_rows) : nullptr;
     a.dot_rows = dot_rows; a.rows_per_example = d->frames * d->n[1];
 
-    CGCK(cudaMemsetAsync(ws + L.off_sc, 0, L.total - L.off_sc, s));          // scalars and counters
     if (y) {
         // A^H y: the forward call on a zero image with eta = 1
         CGCK(cudaMemsetAsync(ws + L.off_r, 0, L.img_bytes, s));

@@ -173,6 +173,14 @@ GLEAM_API int gleam_dc_prepare(const void* y, const float* mask, const gleam_dim
 GLEAM_API int gleam_dc_forward_prepared(const void* x, const void* y, const void* sens, const float* mask,
                                         float eta, void* out, const gleam_dims* dims);
 
+/* ---- zero-filled SENSE image -----------------------------------------------------------------
+ * out = A^H y = sum_c conj(S_c) F^H (Omega y_c): the image the paper's networks start from (its
+ * Experiments section feeds "zero-filled, SENSE-reconstructed" images).  Evaluated as Eq. 3 on a
+ * zero image with eta = 1; arguments, workspace and errors as for gleam_dc_forward.
+ */
+GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mask, void* out,
+                               const gleam_dims* dims);
+
 /* ---- MoDL data-consistency step (Eq. 7, second line) -------------------------------------------
  *
  *     out = (A^H A + mu I)^{-1} (A^H y + mu z)

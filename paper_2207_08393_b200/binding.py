@@ -32,7 +32,7 @@ EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam
            "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end",
            "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes",
            "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size",
-           "gleam_dc_prepare", "gleam_dc_forward_prepared"]
+           "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_adjoint"]
 
 KERNEL_CLASSES = ["zmap", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
                   "col_inv", "cg_vec"]
@@ -97,6 +97,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_dc_forward_static.restype = i32
         lib.gleam_dc_static_scratch_bytes.argtypes = []
         lib.gleam_dc_static_scratch_bytes.restype = u64
+        lib.gleam_dc_adjoint.argtypes = [vp, vp, vp, vp, dp]
+        lib.gleam_dc_adjoint.restype = i32
         lib.gleam_dc_prepare.argtypes = [vp, vp, dp]
         lib.gleam_dc_prepare.restype = i32
         lib.gleam_dc_forward_prepared.argtypes = [vp, vp, vp, vp, f32, vp, dp]
@@ -178,6 +180,11 @@ def gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, dims: gleam_dims) -> None:
     """grad_in = grad_out - eta A^H A grad_out  (VJP of Eq. 3 with respect to x)."""
     _check(load_library().gleam_dc_vjp(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
                                         ctypes.byref(dims)))
+
+
+def gleam_dc_adjoint(y, sens, mask, out, dims: gleam_dims) -> None:
+    """out = A^H y, the zero-filled SENSE image."""
+    _check(load_library().gleam_dc_adjoint(_addr(y), _addr(sens), _addr(mask), _addr(out), ctypes.byref(dims)))
 
 
 def gleam_dc_prepare(y, mask, dims: gleam_dims) -> None:
@@ -273,6 +280,13 @@ class DataConsistency:
             grad_in = self._torch.empty_like(grad_out)
         gleam_dc_vjp(grad_out, sens, mask, eta, grad_in, self.dims())
         return grad_in
+
+    def adjoint(self, y, sens, mask, out=None):
+        """A^H y, shape (B, T, n0, n1, n2)."""
+        if out is None:
+            out = self._torch.empty(self.shape, dtype=y.dtype, device=y.device)
+        gleam_dc_adjoint(y, sens, mask, out, self.dims())
+        return out
 
     def prepare(self, y, mask):
         """For unrolled iterations with the same y and mask: fills the workspace once; follow with

@@ -426,6 +426,20 @@ GLEAM_API int gleam_dc_vjp(const void* grad_out, const void* sens, const float* 
     return gleam::run(grad_out, nullptr, sens, mask, eta, grad_in, dims);
 }
 
+GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mask, void* out, const gleam_dims* dims) {
+    if (!dims || !y || !sens || !mask || !out) return GLEAM_ERR_NULL_POINTER;
+    if (((uintptr_t)out & 15) != 0) return GLEAM_ERR_BAD_DIMS;
+    int rc = gleam::check_device_ptr(out);
+    if (rc != GLEAM_OK) return rc;
+    uint64_t ws = 0;
+    rc = gleam_dc_workspace_size(dims, &ws);               // validates dims before anything is enqueued
+    if (rc != GLEAM_OK) return rc;
+    if (dims->workspace_bytes < ws) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    const uint64_t img_b = (uint64_t)dims->batch * dims->frames * dims->n[0] * dims->n[1] * dims->n[2] * sizeof(gleam::cf);
+    if (cudaMemsetAsync(out, 0, img_b, (cudaStream_t)dims->stream) != cudaSuccess) return GLEAM_ERR_CUDA;
+    return gleam::run(out, y, sens, mask, 1.0f, out, dims);     // 0 - 1 * A^H (A 0 - y), in place
+}
+
 GLEAM_API int gleam_dc_prepare(const void* y, const float* mask, const gleam_dims* dims) {
     return gleam::run(nullptr, y, nullptr, mask, 0.f, nullptr, dims, gleam::RUN_PREPARE);
 }

@@ -277,3 +277,24 @@ def test_prepared_forward_equals_forward(oracle, case):
     assert_close(xb.cpu().numpy(), xo, x, "prepared chain")
     with pytest.raises(g.GleamError):
         g.gleam_dc_prepare(None, tm, dc_b.dims())
+
+
+@pytest.mark.parametrize("case", [
+    (2, 2, 3, 2, (1, 20, 46), MASK_READOUT_INVARIANT, False),
+    (2, 2, 3, 1, (1, 12, 16), MASK_FULL, True),
+    (3, 1, 3, 1, (6, 64, 32), MASK_READOUT_INVARIANT, True),
+])
+def test_adjoint_is_the_zero_filled_image(oracle, case):
+    """gleam_dc_adjoint = A^H y against the oracle's adjoint operator (pinned by the adjoint identity)."""
+    import torch
+    import paper_2207_08393_b200 as g
+    rank, B, C, T, n, kind, weighted = case
+    d, x, y, sens, mask = problem(rank, B, C, T, n, kind, weighted=weighted, seed=5 + sum(n))
+    dev = torch.device("cuda:0")
+    ty, ts, tm = (torch.from_numpy(a).to(dev) for a in (y, sens, mask))
+    dc = g.DataConsistency(B, C, T, rank, n, 0, kind)
+    got = dc.adjoint(ty, ts, tm).cpu().numpy()
+    ref = oracle.apply_AH(y, sens, mask, d)
+    got = got.astype(np.complex128)
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert rel <= 2e-5 and np.abs(got - ref).max() <= 1e-4 * np.abs(ref).max(), rel

@@ -9,16 +9,10 @@ namespace gleam {
 // the workspace; RUN_APPLY: the step with those tables taken from the workspace as they are.
 enum { RUN_ALL = 0, RUN_PREPARE = 1, RUN_APPLY = 2 };
 
-// Conjugate-gradient direction update folded into the operator's load of x (only where
-// dot_rows_supported): x := r + beta_b x, beta_b = sum(rr[parity ^ 1][b]) / sum(rr[parity][b]) over
-// the first nparts entries of the partial-sum arrays rr[2][B][stride]; x (device, writable) receives
-// the new direction.
-struct CgFuse { const void* r; const double* rr; int nparts, stride, parity, B; };
-
 // out = x - eta A^H (A x - y)   (y == nullptr: out = x - eta A^H A x).  Validates its arguments,
 // enqueues on d->stream, returns GLEAM_OK or a GLEAM_ERR_* code.
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode = RUN_ALL, double* dot_rows = nullptr, const struct CgFuse* cg = nullptr);
+        const gleam_dims* d, int mode = RUN_ALL, double* dot_rows = nullptr);
 
 // dot_rows (device, one double per image row, B*T*n1): the one-pass 2-D kernel also stores
 // Re<x_row, out_row> of every row it writes, so that a caller's inner product <x, out> needs no

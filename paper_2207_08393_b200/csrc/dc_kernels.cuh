@@ -34,11 +34,6 @@ struct RowArgs {
     int RPB;            // rows of a full image (n0*n1)
     long long nrows;    // B*T*rpb
     double* dot_rows;   // ROW_FUSED (warp-resident form): if not null, Re<x, out> of every image row, (B*T*rpb)
-    // ROW_FUSED (warp-resident form, no z), conjugate-gradient direction update folded into the load
-    // of x: if cg_r is not null, x := cg_r + beta_b * x with beta_b = rr_new[b] / rr_old[b] (sums of
-    // the partial-sum arrays cg_rr[2][cg_B][cg_stride], first cg_nparts entries; old = cg_parity),
-    // and the new x is also stored to cg_p (the buffer x points to).
-    const cf* cg_r; cf* cg_p; const double* cg_rr; int cg_nparts, cg_stride, cg_parity, cg_B;
 };
 
 struct ColArgs {

@@ -53,7 +53,7 @@ struct WarpLine {
 
 template <int MODE, bool HAS_Z> __device__ __forceinline__ constexpr bool use_z_slots() { return MODE == ROW_FUSED && HAS_Z; }
 
-template <class P, int WARPS, int MODE, bool HAS_Z, bool CG = false>
+template <class P, int WARPS, int MODE, bool HAS_Z>
 __global__ void __launch_bounds__(WARPS * 32)
 warpline_kernel(const RowArgs a) {
     using WL = WarpLine<P, MODE, HAS_Z>;
@@ -87,8 +87,6 @@ warpline_kernel(const RowArgs a) {
     constexpr bool use_z = (MODE == ROW_FUSED) && HAS_Z;
     constexpr bool use_k = (MODE == ROW_INV) || use_z;
 
-    int beta_b = -1;          // CG: example whose beta this lane's line holds
-    float beta_val = 0.f;
     for (long long g = (long long)blockIdx.x * WARPS + warp; g < ngroups; g += wstride) {
         // ---- element offsets of this lane's line; other lines' offsets come by shuffle ----
         const long long row = g * LW + l;
@@ -155,32 +153,6 @@ warpline_kernel(const RowArgs a) {
         issue_coil(0, 0);
         cp_async_commit();
 
-        cf rreg[CG ? R0 : 1];        // CG: this lane's elements of the residual row
-        if (CG) {
-            if (a0 && row_ok) {
-#pragma unroll
-                for (int m = 0; m < R0; ++m) rreg[CG ? m : 0] = a.cg_r[x_off + j + P::BF0 * m];
-            }
-            // beta of every line's example: the warp adds the partial sums of <r,r> (old and new) in
-            // a fixed order; recomputed only when a line moves on to another example
-#pragma unroll
-            for (int ll = 0; ll < LW; ++ll) {
-                const int bl = __shfl_sync(0xffffffffu, b, ll * TPL);
-                const int have = __shfl_sync(0xffffffffu, beta_b, ll * TPL);
-                const bool ok = __shfl_sync(0xffffffffu, (int)row_ok, ll * TPL) != 0;
-                if (!ok || have == bl) continue;
-                const double* p_old = a.cg_rr + ((size_t)a.cg_parity * a.cg_B + bl) * a.cg_stride;
-                const double* p_new = a.cg_rr + ((size_t)(a.cg_parity ^ 1) * a.cg_B + bl) * a.cg_stride;
-                double s_old = 0.0, s_new = 0.0;
-                for (int i = lane; i < a.cg_nparts; i += 32) { s_old += __ldcg(p_old + i); s_new += __ldcg(p_new + i); }
-                for (int o = 16; o > 0; o >>= 1) {
-                    s_old += __shfl_xor_sync(0xffffffffu, s_old, o);
-                    s_new += __shfl_xor_sync(0xffffffffu, s_new, o);
-                }
-                if (l == ll) { beta_b = bl; beta_val = (s_old > 0.0) ? (float)(s_new / s_old) : 0.f; }
-            }
-        }
-
         cf acc[R0];
         cf xreg[R0];     // ROW_FWD / ROW_INV: x fetched once per group and held in registers
         if (!WL::HAS_X && a0 && row_ok) {
@@ -197,21 +169,6 @@ warpline_kernel(const RowArgs a) {
             cp_async_wait<1>();          // everything but the newest group (coil c+1) has landed
             __syncwarp();
 
-            if (CG && c == 0) {
-                // x := r + beta x on the elements this lane uses (the same ones in every later read),
-                // stored back as the new search direction
-                if (a0 && row_ok) {
-#pragma unroll
-                    for (int m = 0; m < R0; ++m) {
-                        const int e = l * N + j + P::BF0 * m;
-                        const cf pv = sX[e], rv = rreg[CG ? m : 0];
-                        const cf nv = make_float2(fmaf(beta_val, pv.x, rv.x), fmaf(beta_val, pv.y, rv.y));
-                        sX[e] = nv;
-                        a.cg_p[x_off + j + P::BF0 * m] = nv;
-                    }
-                }
-                __syncwarp();
-            }
             const cf* cS = sS + buf * TILE + l * N;
             const cf* cK = sK + buf * KTILE + l * KSTRIDE;
             const cf* gK = use_z ? a.z + k_off + c * k_stride : nullptr;   // this line's compact z row

@@ -266,7 +266,7 @@ bool dot_rows_supported(const gleam_dims* d) {
 }
 
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode, double* dot_rows, const CgFuse* cg) {
+        const gleam_dims* d, int mode, double* dot_rows) {
     if (!d || !mask) return GLEAM_ERR_NULL_POINTER;
     if (mode == RUN_PREPARE) {
         if (!y) return GLEAM_ERR_NULL_POINTER;
@@ -275,8 +275,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         return GLEAM_ERR_NULL_POINTER;
     }
     if (mode == RUN_APPLY && !y) return GLEAM_ERR_NULL_POINTER;
-    if ((dot_rows || cg) && !dot_rows_supported(d)) return GLEAM_ERR_UNIMPLEMENTED;   // callers ask first
-    if (cg && y) return GLEAM_ERR_UNIMPLEMENTED;
+    if (dot_rows && !dot_rows_supported(d)) return GLEAM_ERR_UNIMPLEMENTED;   // callers ask first
     Layout L;
     int rc = make_layout(d, y != nullptr, &L);
     if (rc != GLEAM_OK) return rc;
@@ -360,10 +359,6 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         if (L.rank == 2) {
             ra.mask = mask; ra.z = z; ra.rpb = L.n1; ra.row0 = 0; ra.nrows = L.images * L.n1;
             ra.dot_rows = dot_rows;
-            if (cg) {
-                ra.cg_r = (const cf*)cg->r; ra.cg_p = (cf*)const_cast<void*>(x); ra.cg_rr = cg->rr;
-                ra.cg_nparts = cg->nparts; ra.cg_stride = cg->stride; ra.cg_parity = cg->parity; ra.cg_B = cg->B;
-            }
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
             cf* W = (cf*)(ws + L.off_W);

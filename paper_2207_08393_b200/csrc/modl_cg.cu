@@ -13,8 +13,7 @@
 //     cg_dir  : beta = rr' / rr;  p = r + beta p
 //
 // Where the operator is the one-pass 2-D kernel, that kernel also stores Re<p_row, q_row> of every
-// image row it writes (it holds both in registers at its update step) and forms p = r + beta p of the
-// previous step while it loads p: neither cg_dot nor cg_dir is launched, one small launch per step.
+// image row it writes (it holds both in registers at its update step) and cg_dot is not launched.
 //
 // Inner products: every thread accumulates in double precision, a block reduces in a fixed order
 // and stores one partial sum; the kernel that needs the scalar adds the partial sums of its example
@@ -236,11 +235,7 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
     CGCK(cudaGetLastError());
     for (int k = 0; k < n_iter; ++k) {
         a.parity = k & 1;
-        // q = H p / mu; with the one-pass 2-D operator, p = r + beta p of the previous step happens
-        // in its load of p and <p,q> comes back per row
-        CgFuse fuse{a.r, a.part_rr, (int)nb, CG_MAX_BLOCKS, (k - 1) & 1, L.B};
-        CGRUN(run(a.p, nullptr, sens, mask, -1.0f / mu, ws + L.off_q, &dd, RUN_ALL, dot_rows,
-                  (from_rows && k > 0) ? &fuse : nullptr));
+        CGRUN(run(a.p, nullptr, sens, mask, -1.0f / mu, ws + L.off_q, &dd, RUN_ALL, dot_rows));     // q = H p / mu
         if (from_rows) {
             CGCK(prof_mark(GLEAM_K_CG_VEC, s));
             cg_step_kernel<true><<<grid, CG_THREADS, 0, s>>>(a);
@@ -253,7 +248,7 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
             cg_step_kernel<false><<<grid, CG_THREADS, 0, s>>>(a);
             CGCK(cudaGetLastError());
         }
-        if (k + 1 < n_iter && !from_rows) {
+        if (k + 1 < n_iter) {
             CGCK(prof_mark(GLEAM_K_CG_VEC, s));
             cg_dir_kernel<<<grid, CG_THREADS, 0, s>>>(a);
             CGCK(cudaGetLastError());

@@ -39,20 +39,20 @@ inline cudaError_t launch_row(const RowArgs& a, cudaStream_t s) {
 
 // persistent launch of the warp-resident row kernel: one block per resident slot, warps stride
 // over the line groups
-template <class P, int MODE, bool HAS_Z, bool CG = false>
+template <class P, int MODE, bool HAS_Z>
 inline cudaError_t launch_warpline_z(const RowArgs& a, cudaStream_t s) {
     using WL = WarpLine<P, MODE, HAS_Z>;
     constexpr int WARPS = 1;
     constexpr size_t SMEM = sizeof(cf) * WARPS * WL::WARP_ELEMS_ALIGNED;
     static bool attr_done = false;
     static int slots = 0;
-    cudaError_t e = ensure_smem(warpline_kernel<P, WARPS, MODE, HAS_Z, CG>, SMEM, attr_done);
+    cudaError_t e = ensure_smem(warpline_kernel<P, WARPS, MODE, HAS_Z>, SMEM, attr_done);
     if (e != cudaSuccess) return e;
     if (slots == 0) {
         int dev = 0, sms = 0, per_sm = 0;
         if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warpline_kernel<P, WARPS, MODE, HAS_Z, CG>, WARPS * 32,
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warpline_kernel<P, WARPS, MODE, HAS_Z>, WARPS * 32,
                                                                SMEM)) != cudaSuccess) return e;
         slots = sms * (per_sm > 0 ? per_sm : 1);
     }
@@ -60,16 +60,13 @@ inline cudaError_t launch_warpline_z(const RowArgs& a, cudaStream_t s) {
     long long blocks = (groups + WARPS - 1) / WARPS;
     if (blocks <= 0) return cudaSuccess;
     if (blocks > slots) blocks = slots;
-    warpline_kernel<P, WARPS, MODE, HAS_Z, CG><<<(unsigned)blocks, WARPS * 32, SMEM, s>>>(a);
+    warpline_kernel<P, WARPS, MODE, HAS_Z><<<(unsigned)blocks, WARPS * 32, SMEM, s>>>(a);
     return cudaGetLastError();
 }
 
 template <class P, int MODE>
 inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
     if (MODE == ROW_FUSED && a.z != nullptr) return launch_warpline_z<P, MODE, true>(a, s);
-    if constexpr (MODE == ROW_FUSED) {
-        if (a.cg_r != nullptr) return launch_warpline_z<P, MODE, false, true>(a, s);
-    }
     return launch_warpline_z<P, MODE, false>(a, s);
 }
 

@@ -65,9 +65,10 @@ def call_roofline(w, with_y):
     return nbytes, flops
 
 
-def kernel_work(cls, w, launches_per_call):
+def kernel_work(cls, w, launches_per_call, density=1.0):
     """Algorithmic (bytes, flops) of ONE launch of a kernel class for workload w.
-    Per voxel*coil figures are listed beside each case."""
+    Per voxel*coil figures are listed beside each case; density = sampled fraction of the
+    phase-encode positions (the readout transform of y runs at those only)."""
     W = w.voxel_coils / launches_per_call        # voxel*coils one launch processes
     C = w.coils
     l2 = math.log2
@@ -79,9 +80,9 @@ def kernel_work(cls, w, launches_per_call):
         return W * 16, W * (10 * l2(w.n[1]) + 4)
     if cls == "row_fused":      # read S (8) [+ z (8) in the forward call, averaged] + x/out (16/C)
         return W * (8 + 4 + 16 / C), W * (10 * l2(w.n[2]) + 20)
-    if cls == "col_z":          # read y (8), write z (8)
+    if cls == "col_z":          # read y (8), write z (8), at the sampled positions only
         nro = w.n[1] if w.fft_rank == 2 else w.n[0]
-        return W * 16, W * (5 * l2(nro))
+        return W * 16 * density, W * (5 * l2(nro)) * density
     if cls == "col_mid_full":
         nro = w.n[1] if w.fft_rank == 2 else w.n[0]
         return W * 24, W * (10 * l2(nro) + 6)
@@ -248,6 +249,7 @@ def run_ours(args, w):
     inp, y = make_problem(w, seed_offset=rank)
     tx, tg, ts, tm, ty = (torch.from_numpy(a).to(dev) for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
     dc = g.DataConsistency(w.batch, w.coils, w.frames, w.fft_rank, w.n)
+    density = float(np.count_nonzero(inp["mask"])) / inp["mask"].size
     out = torch.empty_like(tx)
     gin = torch.empty_like(tg)
     stream = torch.cuda.current_stream()
@@ -331,8 +333,9 @@ def run_ours(args, w):
     prof = g.gleam_dc_profile_end()
     kernels = {}
     for cls, (ms, cnt) in prof.items():
-        per_call = cnt / (2.0 * chain * prof_steps)        # launches per call, averaged over forward and vjp
-        nbytes, flops = kernel_work(cls, w, max(per_call, 1e-9))
+        calls = (1.0 if cls in ("zmap", "col_z") else 2.0) * chain * prof_steps    # zmap, col_z: forward calls only
+        per_call = cnt / calls
+        nbytes, flops = kernel_work(cls, w, max(per_call, 1e-9), density)
         avg_s = ms * 1e-3 / cnt
         kernels[cls] = {"launches_per_step": cnt / prof_steps, "ms_per_step": ms / prof_steps, "avg_us": avg_s * 1e6,
                         "gbs": nbytes / avg_s / 1e9, "tflops": flops / avg_s / 1e12}
@@ -571,7 +574,7 @@ def run_modl(args, w):
     prof = g.gleam_dc_profile_end()
     kernels = {}
     for cls, (ms, cnt) in prof.items():
-        nbytes, flops = kernel_work(cls, w, 1.0)         # every launch covers the whole problem
+        nbytes, flops = kernel_work(cls, w, 1.0, float(np.count_nonzero(inp["mask"])) / inp["mask"].size)   # every launch covers the whole problem
         avg_s = ms * 1e-3 / cnt
         kernels[cls] = {"launches_per_step": cnt / prof_steps, "ms_per_step": ms / prof_steps, "avg_us": avg_s * 1e6,
                         "gbs": nbytes / avg_s / 1e9, "tflops": flops / avg_s / 1e12}

@@ -57,6 +57,8 @@ struct ColArgs {
     float scale2;       // COL_MID_FULL: 1 / Ntot;  COL_MID_SEP: 1 / (n1 n2)
 };
 
+constexpr int COLZ_SELF_MAX = 1024;   // COL_Z ranks a mask row of at most this many positions by itself
+
 __device__ __forceinline__ int shift_half(int k, int n) { int h = n >> 1; return k >= n - h ? k - (n - h) : k + h; }
 
 // --------------------------------------------------------------------------------------------
@@ -227,7 +229,7 @@ col_kernel(const ColArgs a) {
     const int tiles = (MODE == COL_Z) ? a.ztiles : (a.es + L - 1) / L;
     const long long o = blockIdx.x / tiles;           // outer index
     int i_base = (int)(blockIdx.x % tiles) * L;
-    if (MODE == COL_Z) {
+    if (MODE == COL_Z && a.zlist != nullptr) {
         // lines are ranks of sampled positions: blocks beyond the sampled count leave at once
         const long long bt0 = (o / ((long long)a.C * a.T)) * a.T + (o % a.T);
         if (i_base >= a.zcount[bt0]) return;
@@ -244,7 +246,40 @@ col_kernel(const ColArgs a) {
 
     cf v[R0], u[RL];
 
-    if (MODE == COL_Z) {
+    if constexpr (MODE == COL_Z) {
+      // Without a rank map from an earlier launch (a.zlist == null; rank 2 with at most
+      // COLZ_SELF_MAX phase-encode positions) the block ranks the sampled positions of its mask
+      // row itself: it lists the source positions sh(q) of the sampled raw k indices q in the
+      // order of q -- the order in which the one-pass row kernel counts them.
+      __shared__ int s_list[COLZ_SELF_MAX];
+      __shared__ unsigned s_bal[COLZ_SELF_MAX / 32];
+      const bool self_ranks = a.zlist == nullptr;
+      int self_cnt = 0;
+      if (self_ranks) {
+          const long long bt0 = (o / ((long long)a.C * a.T)) * a.T + (o % a.T);
+          const float* mk = a.mask + bt0 * a.es;
+          const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+          const int nchunks = (a.es + 31) / 32;
+          // every warp marks the sampled entries of its chunks of 32 raw indices ...
+          for (int c = warp; c < nchunks; c += nwarps) {
+              const int q = c * 32 + lane;
+              const bool on = (q < a.es) && (mk[shift_half(q, a.es)] != 0.f);
+              const unsigned bal = __ballot_sync(0xffffffffu, on);
+              if (lane == 0) s_bal[c] = bal;
+          }
+          __syncthreads();
+          // ... then numbers them behind the entries of the chunks before
+          for (int c = warp; c < nchunks; c += nwarps) {
+              int before = 0;
+              for (int e = 0; e < c; ++e) before += __popc(s_bal[e]);
+              const unsigned bal = s_bal[c];
+              const int q = c * 32 + lane;
+              if ((bal >> lane) & 1u) s_list[before + __popc(bal & ((1u << lane) - 1u))] = shift_half(q, a.es);
+          }
+          for (int e = 0; e < nchunks; ++e) self_cnt += __popc(s_bal[e]);
+          __syncthreads();
+          if (i_base >= self_cnt) return;
+      }
       for (;; i_base += tiles * L, i += tiles * L) {
         // Lines are the sampled phase-encode positions of this unit's (b,t), by rank r.
         // z[r] = (g/sqrt(N_ro N_pe)) (-1)^{n_ro} (-1)^{p} M[p] * Rraw^H( (-1)^{k_ro} y[.., p] ),  p = zlist[r]
@@ -252,12 +287,12 @@ col_kernel(const ColArgs a) {
         const int b = (int)(o / ((long long)a.C * a.T));
         const long long bt = (long long)b * a.T + t;
         const long long pe = a.es;
-        const int cnt = a.zcount[bt];
+        const int cnt = self_ranks ? self_cnt : a.zcount[bt];
         if (i_base >= cnt) return;                      // no tile of sampled ranks left for this block
         const bool ok = i < cnt;
         int p = 0, psign = 0; float mv = 0.f;
         if (ok) {
-            p = a.zlist[bt * pe + i];
+            p = self_ranks ? s_list[i] : a.zlist[bt * pe + i];
             mv = a.mask[bt * pe + p];
             psign = (a.rank == 2) ? (p & 1) : ((p / a.n2 + p % a.n2) & 1);
         }

@@ -335,7 +335,10 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             const int zry = (zpair && zpair->ry <= ZMAP_MAX_RY) ? zpair->ry : 0;
             int* zchunk = (int*)(ws + L.off_zchunk);
             const dim3 zgrid((unsigned)((pe + ZMAP_CHUNK - 1) / ZMAP_CHUNK), (unsigned)L.images);
-            if (mode != RUN_APPLY) {      // RUN_APPLY: the tables of an earlier RUN_PREPARE are in the workspace
+            // rank 2 with a one-pass row kernel that counts the sampled positions itself: nothing
+            // but the z table needs the ranks, and the kernel that writes it derives them per block
+            const bool self_ranks = L.rank == 2 && op2->row_is_warp_resident && pe <= COLZ_SELF_MAX;
+            if (mode != RUN_APPLY && !self_ranks) {      // RUN_APPLY: the tables of an earlier RUN_PREPARE are in the workspace
                 CK(prof_mark(GLEAM_K_PREP_M2, s));
                 if (zgrid.x > 1) {        // a table of one chunk needs no counts of earlier chunks
                     zmap_kernel<<<zgrid, ZMAP_THREADS, 0, s>>>(mask, zidx, zlist, zcount, m2c, zstart, zchunk, 1, L.n1, L.n2, L.rank, zry);
@@ -349,6 +352,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             ra.zidx = zidx;
             ColArgs cz = ca;
             cz.y = (const cf*)y; cz.z = z; cz.mask = mask;
+            if (self_ranks) { cz.zlist = nullptr; cz.zcount = nullptr; cz.zidx = nullptr; }
             cz.es = (int)pe; cz.nouter = L.units;
             const int nro = (L.rank == 2) ? L.n1 : L.n0;
             float g = gsign(nro) * gsign(L.n2) * (L.rank == 3 ? gsign(L.n1) : 1.f);

@@ -14,9 +14,11 @@ struct SizeOps {
     cudaError_t (*col)(int mode, const ColArgs& a, cudaStream_t s);
 };
 
+// static_bytes: statically declared shared memory of the kernel, which counts against the same
+// 48 KB default limit as the dynamic part
 template <class K>
-inline cudaError_t ensure_smem(K kernel, size_t bytes, bool& done) {
-    if (!done && bytes > 48 * 1024) {
+inline cudaError_t ensure_smem(K kernel, size_t bytes, bool& done, size_t static_bytes = 0) {
+    if (!done && bytes + static_bytes > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
         if (e != cudaSuccess) return e;
     }
@@ -74,14 +76,17 @@ template <class P, int L, int MODE>
 inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
     using E = LineFFT<P, true, L>;
     static bool attr_done = false;
-    cudaError_t e = ensure_smem(col_kernel<P, L, MODE>, E::SMEM_BYTES, attr_done);
+    cudaError_t e = ensure_smem(col_kernel<P, L, MODE>, E::SMEM_BYTES, attr_done,
+                                MODE == COL_Z ? (COLZ_SELF_MAX + COLZ_SELF_MAX / 32) * sizeof(int) : 0);
     if (e != cudaSuccess) return e;
     long long tiles = (a.es + L - 1) / L;
     ColArgs b = a;
     if (MODE == COL_Z) {
         // the number of sampled ranks is known only on the device: launch a bounded number of blocks
         // per outer index and let them stride over the tiles
-        const long long cap = 4096 / (a.nouter > 0 ? a.nouter : 1) + 16;
+        long long cap = 4096 / (a.nouter > 0 ? a.nouter : 1) + 16;
+        // blocks that rank the mask row themselves pay for that once each: about eight per SM in all
+        if (a.zlist == nullptr) cap = (1184 + a.nouter - 1) / (a.nouter > 0 ? a.nouter : 1);
         if (tiles > cap) tiles = cap;
         b.ztiles = (int)tiles;
     }

@@ -14,6 +14,8 @@
 #include "fft_line.cuh"
 #include <stdint.h>
 
+#include "launch_overlap.cuh"
+
 namespace gleam {
 
 enum RowMode { ROW_FUSED = 0, ROW_FWD = 1, ROW_INV = 2 };
@@ -221,6 +223,7 @@ row_kernel(const RowArgs a) {
 template <class P, int L, int MODE>
 __global__ void __launch_bounds__(LineFFT<P, true, L>::THREADS)
 col_kernel(const ColArgs a) {
+    grid_launch_dependents();    // a one-pass row kernel behind this launch may be scheduled early
     using E = LineFFT<P, true, L>;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL;
     extern __shared__ float2 smem[];

@@ -56,6 +56,8 @@ template <int MODE, bool HAS_Z> __device__ __forceinline__ constexpr bool use_z_
 template <class P, int WARPS, int MODE, bool HAS_Z>
 __global__ void __launch_bounds__(WARPS * 32)
 warpline_kernel(const RowArgs a) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     using WL = WarpLine<P, MODE, HAS_Z>;
     constexpr int KCAP = WL::KCAP, KTILE = WL::KTILE, KSTRIDE = WL::KSTRIDE;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL, TPL = WL::TPL, LW = WL::LW, TILE = WL::TILE;

@@ -62,8 +62,9 @@ inline cudaError_t launch_warpline_z(const RowArgs& a, cudaStream_t s) {
     long long blocks = (groups + WARPS - 1) / WARPS;
     if (blocks <= 0) return cudaSuccess;
     if (blocks > slots) blocks = slots;
-    warpline_kernel<P, WARPS, MODE, HAS_Z><<<(unsigned)blocks, WARPS * 32, SMEM, s>>>(a);
-    return cudaGetLastError();
+    // one round (every warp takes a single group of lines): the launch may overlap the end of the one before
+    return launch_overlapped(groups <= slots, warpline_kernel<P, WARPS, MODE, HAS_Z>, dim3((unsigned)blocks),
+                             dim3(WARPS * 32), SMEM, s, a);
 }
 
 template <class P, int MODE>

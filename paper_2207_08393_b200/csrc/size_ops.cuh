@@ -148,8 +148,7 @@ struct SizeImpl {
     }
     static cudaError_t col(int mode, const ColArgs& a, cudaStream_t s) {
         switch (mode) {
-            // the sampled columns are scattered, so narrow tiles lose no coalescing and give more blocks
-            case COL_Z:        return launch_col<PC, (LC >= 4 ? LC / 4 : 1), COL_Z>(a, s);
+            case COL_Z:        return launch_col<PC, LC, COL_Z>(a, s);
             case COL_MID_SEP:
                 if constexpr (ColPipe<PC, LC>::ELIGIBLE) return launch_colpipe<PC, LC>(a, s);
                 else return launch_col<PC, LC, COL_MID_SEP>(a, s);

@@ -248,6 +248,55 @@ def test_rank3_chunked_workspace_matches_whole_volume(oracle, tmp_path):
     assert np.array_equal(res["out"], whole)
 
 
+def _in_place_chain(x, y, sens, mask, eta, iters):
+    """iters forward calls, then iters VJP calls, all in place on one buffer and enqueued back to
+    back with no synchronisation in between; returns the buffer after each half."""
+    import torch
+    import paper_2207_08393_b200 as g
+    dev = torch.device("cuda:0")
+    tx, ty, ts, tm = (torch.from_numpy(a).to(dev) for a in (x, y, sens, mask))
+    B, T, C, n = x.shape[0], x.shape[1], sens.shape[1], x.shape[2:]
+    dc = g.DataConsistency(B, C, T, 2, n, 0, MASK_READOUT_INVARIANT)
+    for _ in range(iters):
+        dc.forward(tx, ty, ts, tm, eta, tx)
+    after_fwd = tx.clone()
+    for _ in range(iters):
+        dc.vjp(tx, ts, tm, eta, tx)
+    torch.cuda.synchronize()
+    return after_fwd.cpu().numpy(), tx.cpu().numpy()
+
+
+def test_overlapped_launches_equal_serialised_launches(oracle, tmp_path):
+    """One-round launches of the one-pass row kernel start while the launch before them drains and
+    wait for it on the device.  A chain of in-place calls (every call reads what the call before it
+    wrote, and overwrites what that call read) must give the bits of a child process in which
+    every launch is fully serialised (GLEAM_NO_OVERLAP=1, read once per process), and both must
+    match the oracle."""
+    import os
+    import subprocess
+    import sys
+    d, x, y, sens, mask = problem(2, 1, 4, 6, (1, 48, 160), MASK_READOUT_INVARIANT, seed=5, density=0.2)
+    eta, iters = 0.2, 6
+    fwd, vjp = _in_place_chain(x, y, sens, mask, eta, iters)
+    xo = x
+    for _ in range(iters):
+        xo = oracle.dc_forward(xo, y, sens, mask, eta, d).astype(np.complex64)
+    assert_close(fwd, xo, x, "in-place forward chain")
+    np.savez(tmp_path / "in.npz", x=x, y=y, sens=sens, mask=mask)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import sys, numpy as np; sys.path.insert(0, %r)\n"
+        "from tests.test_gpu_parity import _in_place_chain\n"
+        "z = np.load(%r)\n"
+        "fwd, vjp = _in_place_chain(z['x'], z['y'], z['sens'], z['mask'], %r, %d)\n"
+        "np.savez(%r, fwd=fwd, vjp=vjp)\n"
+    ) % (root, str(tmp_path / "in.npz"), eta, iters, str(tmp_path / "out.npz"))
+    subprocess.run([sys.executable, "-c", code], check=True, env=dict(os.environ, GLEAM_NO_OVERLAP="1"), timeout=600)
+    res = np.load(tmp_path / "out.npz")
+    assert np.array_equal(res["fwd"], fwd)
+    assert np.array_equal(res["vjp"], vjp)
+
+
 @pytest.mark.parametrize("case", [
     (2, 2, 3, 2, (1, 20, 46), MASK_READOUT_INVARIANT),
     (2, 1, 4, 1, (1, 64, 320), MASK_READOUT_INVARIANT),      # three-stage plan on the contiguous axis (fallback row kernel)

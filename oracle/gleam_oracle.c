@@ -33,6 +33,12 @@
  * pins are in tests/test_oracle_modl.py (closed form for A^H A = I, dense solve, Krylov-space
  * minimiser for the truncated iteration).
  *
+ * Further down: the gradients of the step with respect to eta and y (oracle_dc_grad_eta,
+ * oracle_dc_grad_y) and the bridge to the learned prior (two-channel layout, complex l1 loss); their
+ * pins are in tests/test_oracle_bridge.py (dense-matrix brute force, exact difference quotients of
+ * oracle_dc, an independent library routine for the layout, closed forms and central differences
+ * for the loss).
+ *
  * Pins (tests/test_oracle_pins.py): brute-force DFT, closed-form spectra of deltas and
  * constants, Parseval, adjoint identity, Hermitian/PSD normal operator, A^H A = I for a full mask
  * and unit-norm sensitivities, affine structure, an independent library FFT.
@@ -556,6 +562,93 @@ int oracle_modl_cg_vjp(const float* g, const float* sens, const float* mask, dou
     const int rc = cg_solve(b, sens, mask, &o, mu, n_iter, out, nthreads);
     free(b);
     return rc;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Gradients of the data-consistency step (Eq. 3) with respect to its two other inputs, for a
+ * cotangent g of the output (conjugate-Wirtinger convention, as for the vector-Jacobian product
+ * with respect to x).  out = x - eta A^H (A x - y) is linear in eta and affine in y, so both are
+ * exact:
+ *     d out / d eta = -A^H (A x - y)     =>   grad_eta[b] = -Re < g_b , A^H (A x - y)_b >
+ *     d out / d y   = +eta A^H           =>   grad_y      = eta A g = eta Omega F S g
+ * < u, v > = sum conj(u) v over the frames and voxels of batch example b.  One value per example:
+ * a step size shared by the batch takes their sum.
+ * ------------------------------------------------------------------------------------------ */
+int oracle_dc_grad_eta(const float* g, const float* x, const float* y, const float* sens, const float* mask,
+                       const int64_t* dims, double* grad_eta, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK || !g || !x || !y || !sens || !mask || !grad_eta) return ORACLE_ERR_ARG;
+    const int64_t n = o.B * o.T * o.V, nk = o.B * o.C * o.T * o.V;
+    zc* k = (zc*)malloc(sizeof(zc) * (size_t)nk);
+    zc* a = (zc*)malloc(sizeof(zc) * (size_t)n);
+    if (!k || !a) { free(k); free(a); return ORACLE_ERR_MEM; }
+    int rc = oracle_apply_A(x, sens, mask, dims, k, nthreads);                  /* k = A x */
+    for (int64_t i = 0; i < nk; ++i) k[i] -= (double)y[2 * i] + I * (double)y[2 * i + 1];   /* A x - y */
+    if (rc == ORACLE_OK) rc = oracle_apply_AH(k, sens, mask, dims, a, nthreads);   /* a = A^H (A x - y) */
+    const int64_t ne = o.T * o.V;
+    for (int64_t b = 0; b < o.B; ++b) {
+        double acc = 0.0;
+        for (int64_t i = b * ne; i < (b + 1) * ne; ++i) {
+            const zc gv = (double)g[2 * i] + I * (double)g[2 * i + 1];
+            acc += creal(conj(gv) * a[i]);
+        }
+        grad_eta[b] = -acc;
+    }
+    free(k); free(a);
+    return rc;
+}
+
+int oracle_dc_grad_y(const float* g, const float* sens, const float* mask, double eta, const int64_t* dims,
+                     zc* grad_y, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK || !g || !sens || !mask || !grad_y) return ORACLE_ERR_ARG;
+    const int rc = oracle_apply_A(g, sens, mask, dims, grad_y, nthreads);       /* A g */
+    const int64_t nk = o.B * o.C * o.T * o.V;
+    for (int64_t i = 0; i < nk; ++i) grad_y[i] *= eta;
+    return rc;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Bridge to the learned prior.  The paper's networks take a complex image as two real channels
+ * (real part, imaginary part) and are trained with an l1 loss on complex images (Implementation /
+ * Training).  Readings: the channel axis sits right after the batch axis,
+ *      complex (B, T, n0, n1, n2)   <->   real (B, 2, T, n0, n1, n2),  channel 0 = Re, 1 = Im;
+ * the loss is the mean modulus of the difference over all B T V complex elements,
+ *      L = (1 / N) sum_i | x_i - r_i | ;
+ * its gradient in the conjugate-Wirtinger convention (the one a real loss back-propagates through
+ * complex tensors, 2 dL/d conj(x)) is (x_i - r_i) / |x_i - r_i| / N, and zero where x_i = r_i.
+ * ------------------------------------------------------------------------------------------ */
+void oracle_complex_to_channels(const float* x, int64_t B, int64_t inner, float* out)
+{
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t i = 0; i < inner; ++i) {
+            out[(b * 2 + 0) * inner + i] = x[2 * (b * inner + i)];
+            out[(b * 2 + 1) * inner + i] = x[2 * (b * inner + i) + 1];
+        }
+}
+
+void oracle_channels_to_complex(const float* ch, int64_t B, int64_t inner, float* out)
+{
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t i = 0; i < inner; ++i) {
+            out[2 * (b * inner + i)] = ch[(b * 2 + 0) * inner + i];
+            out[2 * (b * inner + i) + 1] = ch[(b * 2 + 1) * inner + i];
+        }
+}
+
+/* mean | x - r | over n complex elements; grad (optional, n complex doubles) as stated above */
+double oracle_l1_loss(const float* x, const float* r, int64_t n, zc* grad)
+{
+    double sum = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        const zc d = ((double)x[2 * i] - (double)r[2 * i]) + I * ((double)x[2 * i + 1] - (double)r[2 * i + 1]);
+        const double m = cabs(d);
+        sum += m;
+        if (grad) grad[i] = (m > 0.0) ? d / m / (double)n : 0.0;
+    }
+    return sum / (double)n;
 }
 
 int oracle_max_threads(void)

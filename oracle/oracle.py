@@ -58,6 +58,16 @@ def _load():
         lib.oracle_modl_cg.restype = i32
         lib.oracle_modl_cg_vjp.argtypes = [p, p, p, dbl, i32, p, p, i32]
         lib.oracle_modl_cg_vjp.restype = i32
+        lib.oracle_dc_grad_eta.argtypes = [p, p, p, p, p, p, p, i32]
+        lib.oracle_dc_grad_eta.restype = i32
+        lib.oracle_dc_grad_y.argtypes = [p, p, p, dbl, p, p, i32]
+        lib.oracle_dc_grad_y.restype = i32
+        lib.oracle_complex_to_channels.argtypes = [p, i64, i64, p]
+        lib.oracle_complex_to_channels.restype = None
+        lib.oracle_channels_to_complex.argtypes = [p, i64, i64, p]
+        lib.oracle_channels_to_complex.restype = None
+        lib.oracle_l1_loss.argtypes = [p, p, i64, p]
+        lib.oracle_l1_loss.restype = dbl
         lib.oracle_max_threads.argtypes = []
         lib.oracle_max_threads.restype = i32
         _lib = lib
@@ -240,3 +250,52 @@ def modl_cg_vjp(g, sens, mask, mu: float, n_iter: int, d: Dims, nthreads: int = 
                                     nthreads)
     assert rc == 0, rc
     return out
+
+
+def dc_grad_eta(g, x, y, sens, mask, d: Dims, nthreads: int = 1) -> np.ndarray:
+    """Gradient of Eq. 3 with respect to the step size for a cotangent g of the output, one value
+    per batch example: -Re<g_b, A^H(A x - y)_b>."""
+    g = _c64(g, d.image_shape()); x = _c64(x, d.image_shape()); y = _c64(y, d.kspace_shape())
+    sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
+    out = np.empty(d.batch, dtype=np.float64)
+    dd = d.as_array()
+    rc = _load().oracle_dc_grad_eta(_ptr(g), _ptr(x), _ptr(y), _ptr(sens), _ptr(mask), _ptr(dd), _ptr(out), nthreads)
+    assert rc == 0, rc
+    return out
+
+
+def dc_grad_y(g, sens, mask, eta: float, d: Dims, nthreads: int = 1) -> np.ndarray:
+    """Gradient of Eq. 3 with respect to the measurements: eta Omega F S g, shape of y."""
+    g = _c64(g, d.image_shape()); sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
+    out = np.empty(d.kspace_shape(), dtype=np.complex128)
+    dd = d.as_array()
+    rc = _load().oracle_dc_grad_y(_ptr(g), _ptr(sens), _ptr(mask), float(eta), _ptr(dd), _ptr(out), nthreads)
+    assert rc == 0, rc
+    return out
+
+
+def complex_to_channels(x) -> np.ndarray:
+    """complex64 (B, ...) -> float32 (B, 2, ...): channel 0 the real part, channel 1 the imaginary part."""
+    x = np.ascontiguousarray(x, dtype=np.complex64)
+    out = np.empty((x.shape[0], 2) + x.shape[1:], dtype=np.float32)
+    inner = int(np.prod(x.shape[1:], dtype=np.int64))
+    _load().oracle_complex_to_channels(_ptr(x), x.shape[0], inner, _ptr(out))
+    return out
+
+
+def channels_to_complex(ch) -> np.ndarray:
+    """float32 (B, 2, ...) -> complex64 (B, ...)."""
+    ch = np.ascontiguousarray(ch, dtype=np.float32)
+    assert ch.shape[1] == 2
+    out = np.empty((ch.shape[0],) + ch.shape[2:], dtype=np.complex64)
+    inner = int(np.prod(ch.shape[2:], dtype=np.int64))
+    _load().oracle_channels_to_complex(_ptr(ch), ch.shape[0], inner, _ptr(out))
+    return out
+
+
+def l1_loss(x, ref, with_grad: bool = False):
+    """mean |x - ref| over all complex elements; with_grad also returns (x - ref)/|x - ref|/N."""
+    x = np.ascontiguousarray(x, dtype=np.complex64); ref = _c64(ref, x.shape)
+    grad = np.empty(x.shape, dtype=np.complex128) if with_grad else None
+    val = float(_load().oracle_l1_loss(_ptr(x), _ptr(ref), x.size, _ptr(grad) if with_grad else None))
+    return (val, grad) if with_grad else val

@@ -393,7 +393,8 @@ col_kernel(const ColArgs a) {
                 const float mv = mk[ps];
                 const float w = mv * mv * a.scale2;
                 if (yy) {
-                    const cf q = yy[ps];
+                    // measurements at unsampled positions are not read (they may hold anything)
+                    const cf q = (mv != 0.f) ? yy[ps] : make_float2(0.f, 0.f);
                     const float f = (par ? -a.scale : a.scale) * mv;
                     u[k] = make_float2(fmaf(w, u[k].x, -f * q.x), fmaf(w, u[k].y, -f * q.y));
                 } else {

@@ -317,7 +317,7 @@ struct PairImpl {
     using RT = RowTile<PZ, RY, BY>;
     static_assert(RT::ELIGIBLE, "pair is not eligible for the row-tile kernels");
     template <bool INV> static cudaError_t rows(const TileArgs& a, long long images, cudaStream_t s) {
-        static bool done = false;
+        static PerDevice done;
         cudaError_t e = ensure_smem(rowtile_kernel<PZ, RY, BY, INV>, RT::SMEM_BYTES, done);
         if (e != cudaSuccess) return e;
         const long long blocks = images * a.G * BY;

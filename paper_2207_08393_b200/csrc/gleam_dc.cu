@@ -266,7 +266,7 @@ bool dot_rows_supported(const gleam_dims* d) {
 }
 
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode, double* dot_rows) {
+        const gleam_dims* d, int mode, double* dot_rows, bool check_only) {
     if (!d || !mask) return GLEAM_ERR_NULL_POINTER;
     if (mode == RUN_PREPARE) {
         if (!y) return GLEAM_ERR_NULL_POINTER;
@@ -308,6 +308,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             overlaps(w, L.total, mask, mask_b) || (y && overlaps(w, L.total, y, ksp_b)))
             return GLEAM_ERR_ALIAS;
     }
+    if (check_only) return GLEAM_OK;          // every argument check has passed; nothing is enqueued
 
     cudaStream_t s = (cudaStream_t)d->stream;
     char* ws = (char*)d->workspace;
@@ -435,10 +436,9 @@ GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mas
     if (((uintptr_t)out & 15) != 0) return GLEAM_ERR_BAD_DIMS;
     int rc = gleam::check_device_ptr(out);
     if (rc != GLEAM_OK) return rc;
-    uint64_t ws = 0;
-    rc = gleam_dc_workspace_size(dims, &ws);               // validates dims before anything is enqueued
+    // all argument checks of the step itself, before the output is cleared
+    rc = gleam::run(out, y, sens, mask, 1.0f, out, dims, gleam::RUN_ALL, nullptr, true);
     if (rc != GLEAM_OK) return rc;
-    if (dims->workspace_bytes < ws) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
     const uint64_t img_b = (uint64_t)dims->batch * dims->frames * dims->n[0] * dims->n[1] * dims->n[2] * sizeof(gleam::cf);
     if (cudaMemsetAsync(out, 0, img_b, (cudaStream_t)dims->stream) != cudaSuccess) return GLEAM_ERR_CUDA;
     return gleam::run(out, y, sens, mask, 1.0f, out, dims);     // 0 - 1 * A^H (A 0 - y), in place
@@ -592,14 +592,18 @@ static int run_host(const void* x, const void* y, const void* sens, const float*
     if (arena_bytes < off[6]) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
     char* a = (char*)arena;
     cudaStream_t s = (cudaStream_t)dims->stream;
+    gleam_dims d = *dims;
+    d.workspace = a + off[5];
+    d.workspace_bytes = sz[5];
+    // argument checks on the staged device pointers come before the first copy is enqueued
+    rc = gleam::run(a + off[0], y ? a + off[1] : nullptr, a + off[2], (const float*)(a + off[3]), eta, a + off[4], &d,
+                    gleam::RUN_ALL, nullptr, true);
+    if (rc != GLEAM_OK) return rc;
     const void* src[4] = {x, y, sens, mask};
     for (int i = 0; i < 4; ++i) {
         if (!src[i]) continue;
         if (cudaMemcpyAsync(a + off[i], src[i], sz[i], cudaMemcpyHostToDevice, s) != cudaSuccess) return GLEAM_ERR_CUDA;
     }
-    gleam_dims d = *dims;
-    d.workspace = a + off[5];
-    d.workspace_bytes = sz[5];
     rc = gleam::run(a + off[0], y ? a + off[1] : nullptr, a + off[2], (const float*)(a + off[3]), eta, a + off[4], &d);
     if (rc != GLEAM_OK) return rc;
     if (cudaMemcpyAsync(out, a + off[4], sz[4], cudaMemcpyDeviceToHost, s) != cudaSuccess) return GLEAM_ERR_CUDA;

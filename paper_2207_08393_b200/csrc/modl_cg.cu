@@ -222,6 +222,8 @@ static int modl_cg(const void* z, const void* y, const void* sens, const float* 
     double* dot_rows = from_rows ? (double*)(ws + L.off_rows) : nullptr;
     a.dot_rows = dot_rows; a.rows_per_example = d->frames * d->n[1];
 
+    // the operator's own argument checks (y, sens, mask) before anything is enqueued
+    CGRUN(run(ws + L.off_r, y, sens, mask, 1.0f, ws + L.off_q, &dd, RUN_ALL, nullptr, true));
     if (y) {
         // A^H y: the forward call on a zero image with eta = 1
         CGCK(cudaMemsetAsync(ws + L.off_r, 0, L.img_bytes, s));

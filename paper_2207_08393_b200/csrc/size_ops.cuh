@@ -5,7 +5,22 @@
 #include "dc_warpline.cuh"
 #include "dc_colpipe.cuh"
 
+#include <atomic>
+
 namespace gleam {
+
+// Launch state that CUDA keeps per device (function attributes, occupancy, SM count) is cached per
+// device ordinal: one process may drive several GPUs, from several host threads.  The cached values
+// are idempotent, so two threads that race on a first use both compute and store the same thing.
+constexpr int MAX_DEVICES = 64;
+struct PerDevice {
+    std::atomic<int> v[MAX_DEVICES];         // 0 = not yet known on that device
+    std::atomic<int>* slot() {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+        return &v[dev];
+    }
+};
 
 struct SizeOps {
     int N;
@@ -17,19 +32,35 @@ struct SizeOps {
 // static_bytes: statically declared shared memory of the kernel, which counts against the same
 // 48 KB default limit as the dynamic part
 template <class K>
-inline cudaError_t ensure_smem(K kernel, size_t bytes, bool& done, size_t static_bytes = 0) {
-    if (!done && bytes + static_bytes > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-        if (e != cudaSuccess) return e;
-    }
-    done = true;
+inline cudaError_t ensure_smem(K kernel, size_t bytes, PerDevice& done, size_t static_bytes = 0) {
+    if (bytes + static_bytes <= 48 * 1024) return cudaSuccess;
+    std::atomic<int>* flag = done.slot();               // null: device ordinal outside the cache, set every time
+    if (flag && flag->load(std::memory_order_acquire)) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return e;
+    if (flag) flag->store(1, std::memory_order_release);
+    return cudaSuccess;
+}
+
+// resident blocks of `kernel` on the current device (SM count x blocks per SM), cached per device
+template <class K>
+inline cudaError_t resident_slots(K kernel, int threads, size_t smem, PerDevice& cache, int* out) {
+    std::atomic<int>* c = cache.slot();
+    if (c) { const int v = c->load(std::memory_order_acquire); if (v > 0) { *out = v; return cudaSuccess; } }
+    int dev = 0, sms = 0, per_sm = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem)) != cudaSuccess) return e;
+    *out = sms * (per_sm > 0 ? per_sm : 1);
+    if (c) c->store(*out, std::memory_order_release);
     return cudaSuccess;
 }
 
 template <class P, int L, int MODE>
 inline cudaError_t launch_row(const RowArgs& a, cudaStream_t s) {
     using E = LineFFT<P, false, L>;
-    static bool attr_done = false;
+    static PerDevice attr_done;
     cudaError_t e = ensure_smem(row_kernel<P, L, MODE>, E::SMEM_BYTES, attr_done);
     if (e != cudaSuccess) return e;
     const long long blocks = (a.nrows + L - 1) / L;
@@ -46,18 +77,12 @@ inline cudaError_t launch_warpline_z(const RowArgs& a, cudaStream_t s) {
     using WL = WarpLine<P, MODE, HAS_Z>;
     constexpr int WARPS = 1;
     constexpr size_t SMEM = sizeof(cf) * WARPS * WL::WARP_ELEMS_ALIGNED;
-    static bool attr_done = false;
-    static int slots = 0;
+    static PerDevice attr_done;
+    static PerDevice slots_cache;
     cudaError_t e = ensure_smem(warpline_kernel<P, WARPS, MODE, HAS_Z>, SMEM, attr_done);
     if (e != cudaSuccess) return e;
-    if (slots == 0) {
-        int dev = 0, sms = 0, per_sm = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warpline_kernel<P, WARPS, MODE, HAS_Z>, WARPS * 32,
-                                                               SMEM)) != cudaSuccess) return e;
-        slots = sms * (per_sm > 0 ? per_sm : 1);
-    }
+    int slots = 0;
+    if ((e = resident_slots(warpline_kernel<P, WARPS, MODE, HAS_Z>, WARPS * 32, SMEM, slots_cache, &slots)) != cudaSuccess) return e;
     const long long groups = (a.nrows + WL::LW - 1) / WL::LW;
     long long blocks = (groups + WARPS - 1) / WARPS;
     if (blocks <= 0) return cudaSuccess;
@@ -76,7 +101,7 @@ inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
 template <class P, int L, int MODE>
 inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
     using E = LineFFT<P, true, L>;
-    static bool attr_done = false;
+    static PerDevice attr_done;
     cudaError_t e = ensure_smem(col_kernel<P, L, MODE>, E::SMEM_BYTES, attr_done,
                                 MODE == COL_Z ? (COLZ_SELF_MAX + COLZ_SELF_MAX / 32) * sizeof(int) : 0);
     if (e != cudaSuccess) return e;
@@ -102,18 +127,12 @@ inline cudaError_t launch_col(const ColArgs& a, cudaStream_t s) {
 template <class P, int L, bool HAS_Z>
 inline cudaError_t launch_colpipe_z(const ColArgs& a, cudaStream_t s) {
     using CP = ColPipe<P, L>;
-    static bool attr_done = false;
-    static int slots = 0;
+    static PerDevice attr_done;
+    static PerDevice slots_cache;
     cudaError_t e = ensure_smem(colpipe_mid_sep_kernel<P, L, HAS_Z>, CP::SMEM_BYTES, attr_done);
     if (e != cudaSuccess) return e;
-    if (slots == 0) {
-        int dev = 0, sms = 0, per_sm = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, colpipe_mid_sep_kernel<P, L, HAS_Z>, CP::THREADS,
-                                                               CP::SMEM_BYTES)) != cudaSuccess) return e;
-        slots = sms * (per_sm > 0 ? per_sm : 1);
-    }
+    int slots = 0;
+    if ((e = resident_slots(colpipe_mid_sep_kernel<P, L, HAS_Z>, CP::THREADS, CP::SMEM_BYTES, slots_cache, &slots)) != cudaSuccess) return e;
     const long long tiles_per_o = (a.es + L - 1) / L;
     const long long tiles = a.nouter * tiles_per_o;
     if (tiles <= 0) return cudaSuccess;

@@ -101,20 +101,35 @@ def test_single_coil_single_everything(oracle):
     check(oracle, d, x, y, sens, mask, 0.5, what="2x2")
 
 
-def test_unsampled_measurements_are_never_read(oracle):
-    d, x, y, sens, mask = problem(2, 1, 3, 1, (1, 16, 24), MASK_READOUT_INVARIANT, seed=8)
-    ref = oracle.dc_forward(x, y * mask[:, None, :, None, None, :], sens, mask, 1.0, d)
+@pytest.mark.parametrize("rank,n", [(2, (1, 16, 24)), (3, (6, 10, 12))])
+@pytest.mark.parametrize("mask_kind", [MASK_READOUT_INVARIANT, MASK_FULL])
+def test_unsampled_measurements_are_never_read(oracle, rank, n, mask_kind):
+    """y may hold anything (here NaN) wherever the mask is zero, for both mask kinds and ranks."""
+    d, x, y, sens, mask = problem(rank, 1, 3, 1, n, mask_kind, seed=8 + rank + mask_kind)
+    dfull = Dims(1, 3, 1, rank, n, 0, MASK_FULL)
+    mfull = np.broadcast_to(mask.reshape(mask.shape[:2] + (1,) * (5 - mask.ndim) + mask.shape[2:]), dfull.mask_shape())
+    y_clean = y * mfull[:, None]
+    ref = oracle.dc_forward(x, y_clean, sens, mask, 1.0, d)
     y_bad = y.copy()
-    y_bad[..., mask[0, 0] == 0] = np.nan
-    got = run_gpu(x, y_bad, sens, mask, 1.0, 2, 0, MASK_READOUT_INVARIANT)
+    y_bad[np.broadcast_to(mfull[:, None] == 0, y.shape)] = np.nan
+    got = run_gpu(x, y_bad, sens, mask, 1.0, rank, 0, mask_kind)
     assert_close(got, ref, x, "NaN in unsampled y")
 
 
-def test_deterministic_across_repeats():
-    d, x, y, sens, mask = problem(2, 2, 8, 1, (1, 64, 160), MASK_READOUT_INVARIANT, seed=9)
-    first = run_gpu(x, y, sens, mask, 1.0, 2, 0, MASK_READOUT_INVARIANT)
-    for _ in range(5):
-        assert np.array_equal(first, run_gpu(x, y, sens, mask, 1.0, 2, 0, MASK_READOUT_INVARIANT))
+@pytest.mark.parametrize("case", [
+    (2, 2, 8, 1, (1, 64, 160), MASK_READOUT_INVARIANT),      # one-pass 2-D kernel
+    (3, 1, 4, 1, (8, 64, 32), MASK_READOUT_INVARIANT),       # separable 3-D path
+    (3, 1, 3, 1, (6, 20, 24), MASK_FULL),                    # general path
+])
+def test_deterministic_across_repeats(case):
+    """No float atomics anywhere: 20 repeats give the same bits (forward and VJP)."""
+    rank, B, C, T, n, kind = case
+    d, x, y, sens, mask = problem(rank, B, C, T, n, kind, seed=9)
+    first = run_gpu(x, y, sens, mask, 1.0, rank, 0, kind)
+    first_v = run_gpu(x, None, sens, mask, 1.0, rank, 0, kind)
+    for _ in range(20):
+        assert np.array_equal(first, run_gpu(x, y, sens, mask, 1.0, rank, 0, kind))
+        assert np.array_equal(first_v, run_gpu(x, None, sens, mask, 1.0, rank, 0, kind))
 
 
 def test_cross_export_identities():
@@ -160,6 +175,14 @@ def test_error_codes_on_device_buffers():
     assert e.value.status == binding.GLEAM_ERR_ALIAS
     g.gleam_dc_forward(x, y, s, m, 1.0, x, d)                  # exact alias is allowed
     torch.cuda.synchronize()
+    # a call that returns an argument error has enqueued nothing: an adjoint whose out overlaps y
+    # must leave both untouched (it clears out only after every check has passed)
+    y.fill_(3.0)
+    with pytest.raises(g.GleamError) as e:
+        g.gleam_dc_adjoint(y, s, m, y.view(torch.float32)[0, 1].data_ptr(), d)
+    assert e.value.status == binding.GLEAM_ERR_ALIAS
+    torch.cuda.synchronize()
+    assert bool((y == 3.0).all())
 
 
 # ----------------------------------------------------------------------------------------------

@@ -88,6 +88,8 @@ def kernel_work(cls, w, launches_per_call, density=1.0):
         return W * 24, W * (10 * l2(nro) + 6)
     if cls in ("col_fwd", "col_inv"):
         return W * 16, W * (5 * l2(w.n[1]))
+    if cls == "fused3d":        # one launch = the whole call: read S (8) + x (8/C), write out (8/C); both transforms over (n1, n2)
+        return W * (8 + 16 / C), W * (10 * l2(w.n[1] * w.n[2]) + 20)
     if cls == "cg_vec":         # image-sized vector kernels of the CG solve: on average 3.7 passes of 8 B
         return W * (3.7 * 8 / C), W * (8.0 / C)     # per voxel (init 5, dot 2, step 6, dir 3 passes)
     return 0.0, 0.0
@@ -176,12 +178,20 @@ def aggregate(local_ms, local_units, world, dist=None, device=None):
 
 
 # ------------------------------------------------------------------------------------------------
-def reference_sample(w):
-    """Bounded sample of a workload for the CPU oracle: same kind of problem, fewer units."""
+def reference_sample(w, cores=None):
+    """Bounded sample of a workload for the CPU oracle: same kind of problem, fewer units.  With at
+    least 8 host threads the whole workload is the sample (knee3d: about 10 s per step).  A smaller
+    knee3d sample keeps 40 readout slabs, so that the readout axis still goes through the oracle's
+    FFT route (lengths above 32) like the full volume, not through its direct sum."""
     from paper_2207_08393_b200 import workloads as wl
+    if cores is None:
+        from oracle import oracle
+        cores = oracle.max_threads()
     if w.name == "knee3d":
-        return wl.scaled(w, n=(16, w.n[1], w.n[2])), "8 coils, 16 of 320 readout slabs (16x320x256)"
-    if w.name in ("knee2d", "brain2d"):
+        if cores >= 8:
+            return w, "whole workload"
+        return wl.scaled(w, n=(40, w.n[1], w.n[2])), "8 coils, 40 of 320 readout slabs (40x320x256)"
+    if w.name in ("knee2d", "brain2d") and cores < 8:
         return wl.scaled(w, batch=1), "batch 1 of %d" % w.batch
     return w, "whole workload"
 
@@ -200,10 +210,10 @@ def run_reference(args, w):
         return
     from oracle import oracle
     oracle.build()
-    ws, sample_txt = reference_sample(w)
+    cores = oracle.max_threads()
+    ws, sample_txt = reference_sample(w, cores)
     inp, y = make_problem(ws)
     d = oracle.Dims(ws.batch, ws.coils, ws.frames, ws.fft_rank, ws.n, 0, oracle.MASK_READOUT_INVARIANT)
-    cores = oracle.max_threads()
 
     def step():
         oracle.dc_forward(inp["x"], y, inp["sens"], inp["mask"], ws.eta, d, nthreads=cores)
@@ -220,7 +230,9 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "description": w.description, "sample": sample_txt},
+        "config": {"workload": w.name, "description": w.description, "sample": sample_txt,
+                   "step": "%d gleam_dc_forward + %d gleam_dc_vjp evaluated by the oracle" % (1, 1),
+                   "voxel_coils_per_step": ws.voxel_coils},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample_txt},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -246,10 +258,15 @@ def run_ours(args, w):
     g.load_library()
     peaks = load_peaks()
 
+    from paper_2207_08393_b200 import workloads as wl
     inp, y = make_problem(w, seed_offset=rank)
-    tx, tg, ts, tm, ty = (torch.from_numpy(a).to(dev) for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
-    dc = g.DataConsistency(w.batch, w.coils, w.frames, w.fft_rank, w.n)
+    full_mask = args.mask == "full"
+    mask_kind = g.GLEAM_MASK_FULL if full_mask else g.GLEAM_MASK_READOUT_INVARIANT
     density = float(np.count_nonzero(inp["mask"])) / inp["mask"].size
+    if full_mask:        # the same sampling pattern handed over as a general (B, T, n0, n1, n2) mask
+        inp = dict(inp, mask=wl.expand_mask(w, inp["mask"]))
+    tx, tg, ts, tm, ty = (torch.from_numpy(a).to(dev) for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
+    dc = g.DataConsistency(w.batch, w.coils, w.frames, w.fft_rank, w.n, mask_kind=mask_kind)
     out = torch.empty_like(tx)
     gin = torch.empty_like(tg)
     stream = torch.cuda.current_stream()
@@ -276,8 +293,10 @@ def run_ours(args, w):
             src = dst
 
     def step():
-        forward_chain()
-        vjp_chain()
+        if args.calls != "vjp":
+            forward_chain()
+        if args.calls != "forward":
+            vjp_chain()
 
     flush = None
     inputs_bytes = sum(t.numel() * t.element_size() for t in (tx, tg, ts, tm, ty))
@@ -322,6 +341,16 @@ def run_ours(args, w):
     t_end = time.time()
     total_ms, total_units = aggregate(local_ms, w.voxel_coils * chain * args.steps, world, dist, dev)
     value = total_units / (total_ms * 1e-3)
+    if args.kernels_only:
+        if sampler:
+            sampler.stop()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "workload": w.name, "calls": args.calls, "steps": args.steps,
+                              "ms_per_step": total_ms / args.steps, "gpu_launches": int(launches), "profiler_run": True,
+                              "fused_wait_us_last_call": g.gleam_dc_fused_wait_stats(dc.dims())}))
+        if dist is not None:
+            dist.destroy_process_group()
+        return
 
     # ---- per-kernel pass (CUDA events around every launch, on the launching stream) ----------
     prof_steps = min(args.steps, 5)
@@ -353,7 +382,7 @@ def run_ours(args, w):
 
     # ---- the same chain with the y-dependent tables computed once per step (gleam_dc_prepare) ----
     prepared = None
-    if chain > 1:
+    if chain > 1 and not full_mask:
         def forward_chain_prepared():
             dc.prepare(ty, tm)
             src = tx
@@ -377,13 +406,26 @@ def run_ours(args, w):
                     "value": w.voxel_coils * chain / (step_ms * 1e-3), "unit": UNIT,
                     "what": "1 gleam_dc_prepare + %d gleam_dc_forward_prepared per step, VJP chain as in the main number" % chain}
 
+    # ---- the same steps without the L2 flush (problems that fit in L2: both figures are reported) ----
+    warm = None
+    if flush is not None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        step(); torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream); torch.cuda.synchronize()
+        wms = e0.elapsed_time(e1) / args.steps
+        warm = {"ms_per_step": wms, "value": w.voxel_coils * chain / (wms * 1e-3), "unit": UNIT,
+                "what": "steps back to back, inputs and tables left in L2 by the step before (rank 0)"}
+
     clocks = sampler.stop(t_begin, t_end) if sampler else None
 
     # ---- end to end through the host-buffer entry points --------------------------------------
     e2e_steps = max(1, min(args.steps, 3 if inputs_bytes > (1 << 30) else 10))
     hx, hg, hs, hm, hy = (torch.from_numpy(a).pin_memory() for a in (inp["x"], inp["g"], inp["sens"], inp["mask"], y))
     hout, hgin = torch.empty_like(hx).pin_memory(), torch.empty_like(hg).pin_memory()
-    d_host = g.make_dims(w.batch, w.coils, w.frames, w.fft_rank, w.n, stream=stream)
+    d_host = g.make_dims(w.batch, w.coils, w.frames, w.fft_rank, w.n, mask_kind=mask_kind, stream=stream)
     arena = torch.empty(g.gleam_dc_host_arena_size(d_host), dtype=torch.uint8, device=dev)
 
     def step_host():
@@ -424,7 +466,7 @@ def run_ours(args, w):
     else:
         roof = {"bound": "alu", "achieved": kd["tflops"], "peak": alu_peak, "unit": "TFLOP/s", "frac": t_alu}
     roof.update({"kernel": dom, "peak_source": peaks["source"] + (" copy bandwidth" if roof["bound"] == "hbm" else
-                 " sm_max_mhz x 148 SMs x 128 lanes x 2"), "traffic": TRAFFIC.get((w.name, dom)),
+                 " sm_max_mhz x 148 SMs x 128 lanes x 2"), "traffic": measured_traffic(w.name, dom),
                  "share_of_step": kd["ms_per_step"] / sum(k["ms_per_step"] for k in kernels.values())})
     ns = {}
     for name, with_y, ms in (("forward", True, split[0]), ("vjp", False, split[1])):
@@ -439,12 +481,15 @@ def run_ours(args, w):
         from oracle import oracle
         oracle.build()
         cores = oracle.max_threads()
-        wsamp, sample_txt = (w, "whole workload, 1 step") if w.name != "knee3d" or cores >= 8 else reference_sample(w)
+        wsamp, sample_txt = (w, "whole workload, 1 step") if w.name != "knee3d" or cores >= 8 else reference_sample(w, cores)
         if wsamp is not w:
             inp_c, y_c = make_problem(wsamp)
+            if full_mask:
+                inp_c = dict(inp_c, mask=wl.expand_mask(wsamp, inp_c["mask"]))
         else:
             inp_c, y_c = inp, y
-        d = oracle.Dims(wsamp.batch, wsamp.coils, wsamp.frames, wsamp.fft_rank, wsamp.n, 0, oracle.MASK_READOUT_INVARIANT)
+        d = oracle.Dims(wsamp.batch, wsamp.coils, wsamp.frames, wsamp.fft_rank, wsamp.n, 0,
+                        oracle.MASK_FULL if full_mask else oracle.MASK_READOUT_INVARIANT)
         t0 = time.perf_counter()
         oracle.dc_forward(inp_c["x"], y_c, inp_c["sens"], inp_c["mask"], wsamp.eta, d, nthreads=cores)
         oracle.dc_vjp(inp_c["g"], inp_c["sens"], inp_c["mask"], wsamp.eta, d, nthreads=cores)
@@ -458,7 +503,8 @@ def run_ours(args, w):
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "description": w.description, "step": "%d chained gleam_dc_forward + %d chained gleam_dc_vjp" % (chain, chain),
                    "voxel_coils_per_step": w.voxel_coils * chain, "e2e_step": "1 forward + 1 vjp with host buffers", "parallelism": "replicas only" if world > 1 else "1 gpu",
-                   "l2": "inputs exceed L2" if flush is None else "256 MB L2 flush before every step (chain)"},
+                   "l2": "inputs exceed L2" if flush is None else "256 MB L2 flush before every step (chain)",
+                   "mask": "general (B,T,n0,n1,n2) array" if full_mask else "readout-invariant"},
         "ms_per_iteration": total_ms / args.steps / chain,
         "clocks": clocks,
         "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -467,6 +513,7 @@ def run_ours(args, w):
         "roofline": roof,
         "call_roofline": ns,
         "prepared_chain": prepared,
+        "warm_l2": warm,
         "kernels": kernels,
         "cpu_baseline": cpu,
     }
@@ -654,14 +701,29 @@ def run_modl(args, w):
     if dist is not None:
         dist.destroy_process_group()
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
-# an ncu capture, keyed by (workload, kernel class); None until a capture of the current kernel exists.
-TRAFFIC = {
-    # rowtile_kernel<Plan<256,16,16>,16,20,INV>, whole-volume launches of knee3d (1-pass ncu capture of
-    # bench.py itself, profiles/rowtile_knee3d.md): dram read + write per launch
-    ("knee3d", "row_inv"): 3.57e9 + 0.203e9,
-    ("knee3d", "row_fwd"): 1.89e9 + 1.63e9,
-}
+def kernel_sources_digest():
+    """SHA-256 over the CUDA sources of the library: identifies the kernels a counter capture was taken on."""
+    import hashlib
+    csrc = os.path.join(ROOT, "paper_2207_08393_b200", "csrc")
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(csrc)):
+        h.update(name.encode())
+        h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()
+
+
+def measured_traffic(workload, kernel):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel class from the
+    recorded ncu captures; None when there is no capture or the kernel sources have changed since."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path))
+    digest = kernel_sources_digest()
+    for e in rec.get("captures", []):
+        if e.get("workload") == workload and e.get("kernel") == kernel and e.get("sources_sha256") == digest:
+            return float(e["dram_bytes_per_launch"])
+    return None
 
 
 def main():
@@ -672,6 +734,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="knee3d")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mask", default="invariant", choices=["invariant", "full"],
+                    help="invariant: the mask is handed over in readout-invariant form (separable path); full: the same "
+                         "pattern as a general (B,T,n0,n1,n2) array (arbitrary-mask path)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="profiler run: warm-up and timed steps only, then a short JSON line (no per-kernel pass, no "
+                         "end-to-end leg, no CPU baseline)")
+    ap.add_argument("--calls", default="both", choices=["both", "forward", "vjp"], help="which calls a step makes")
+    ap.add_argument("--print-sources-digest", action="store_true", help="print the digest that keys profiles/dram_traffic.json")
     ap.add_argument("--method", default="dc", choices=["dc", "modl"],
                     help="dc: the gradient data-consistency step (Eq. 3); modl: the model inversion of Eq. 7 "
                          "by 10 conjugate-gradient steps (use with --workload knee2d or cine)")
@@ -679,7 +749,16 @@ def main():
     ap.add_argument("--cg-steps", type=int, default=10)
     args = ap.parse_args()
     from paper_2207_08393_b200 import workloads as wl
-    w = wl.WORKLOADS[args.workload]
+    if args.print_sources_digest:
+        print(kernel_sources_digest())
+        return
+    if args.workload == "knee3d_small":
+        # profiler case: the full 320 x 256 phase-encode plane of knee3d (same kernels and launch shapes), 20 of
+        # the 320 readout slabs: 0.4 GB on the device, larger than L2, small enough for multi-pass counter captures
+        w = wl.scaled(wl.WORKLOADS["knee3d"], name="knee3d_small", n=(20, 320, 256),
+                      description="profiler case: knee3d with 20 of 320 readout slabs (8 coils, 20x320x256)")
+    else:
+        w = wl.WORKLOADS[args.workload]
     if args.method == "modl":
         run_modl(args, w)
     elif args.impl == "reference":

@@ -112,6 +112,42 @@ GLEAM_API int gleam_dc_vjp(const void* grad_out, const void* sens, const float* 
 GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes);
 
 /*
+ * Device-side status of the work enqueued so far with these dims and this workspace (the paper has
+ * no counterpart).  The separable 3-D path (fft_rank 3, readout-invariant mask, n2 = 256 and n1 a
+ * compiled multiple of 16) runs Eq. 3 as one persistent kernel whose blocks hand slabs of the coil
+ * workspace to one another through L2; every wait of one block for another is bounded (two seconds).
+ * A wait that runs out makes the kernel stop early and leaves an error word in the workspace.  This
+ * call synchronises dims->stream, reads the word and returns GLEAM_ERR_TIMEOUT if it is set (the
+ * output of that call is then undefined), GLEAM_OK otherwise.  For every other problem class it
+ * only synchronises and returns GLEAM_OK: no other kernel waits on another block.
+ */
+GLEAM_API int gleam_dc_check_status(const gleam_dims* dims);
+
+/*
+ * Selects (on != 0) or deselects the persistent kernel for the problem class described above; the default
+ * is off unless the environment holds GLEAM_FUSED=1, because the three whole-volume passes measure faster
+ * on one B200.  Process-wide; call it before gleam_dc_workspace_size (the scratch layout depends on it).
+ */
+GLEAM_API void gleam_dc_set_fused(int32_t on);
+
+/*
+ * Measurement aid: how long the blocks of the last persistent-kernel call with these dims and workspace
+ * waited, summed over all blocks.  ns_and_counts receives n_kinds (<= 5) pairs {nanoseconds, waits that
+ * had to spin}: 0 a ring slot to become free, 1 the first pass of a slab to complete, 2 the middle pass
+ * to complete (all three: one block waiting for others), 3 and 4 a staged tile (sensitivities / workspace)
+ * that had not landed when a compute group needed it.  Synchronises dims->stream.
+ */
+GLEAM_API int gleam_dc_fused_wait_stats(const gleam_dims* dims, uint64_t* ns_and_counts, int32_t n_kinds);
+
+/*
+ * Test aid for the bounded waits above: the item with this number (>= 0) of the persistent kernel is
+ * drawn but neither run nor counted as done, so that the blocks depending on it run into their wait
+ * limit; wait_limit_ns shortens the limit (0 = the default).  (-1, 0) restores normal operation.
+ * Process-wide; not for production use.
+ */
+GLEAM_API void gleam_dc_debug_fused(int32_t withhold_item, uint64_t wait_limit_ns);
+
+/*
  * GLEAM_OK if a transform of this length is supported along an axis (even lengths whose plan is
  * compiled in), GLEAM_ERR_UNSUPPORTED_SIZE otherwise.
  */
@@ -181,6 +217,25 @@ GLEAM_API int gleam_dc_forward_prepared(const void* x, const void* y, const void
 GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mask, void* out,
                                const gleam_dims* dims);
 
+/* ---- gradients of Eq. 3 with respect to the step size and the measurements --------------------------
+ * out = x - eta A^H (A x - y) is linear in eta and affine in y.  For a cotangent g = grad_out of the
+ * output (conjugate-Wirtinger convention, as for gleam_dc_vjp):
+ *     grad_eta[b] = -Re < g_b , A^H (A x - y)_b >        one double per batch example (device, B values);
+ *                                                        a step size shared by the batch takes their sum
+ *     grad_y      = eta A g = eta Omega F S g             complex64, layout of y; zero where the mask is zero
+ * The paper does not say whether the step size 2t of Eq. 3 is trained; these are the exact derivatives
+ * for a caller that trains it, or that needs the sensitivity of the step to the measurements.
+ * dims->workspace: gleam_dc_grad_workspace_size bytes.  grad_eta evaluates the step once with eta = 1
+ * (all kernels of gleam_dc_forward) and reduces in double precision in a fixed order; grad_y runs the
+ * forward operator alone.  Argument rules and errors as for gleam_dc_forward; nothing may overlap an
+ * output or the workspace.
+ */
+GLEAM_API int gleam_dc_grad_eta(const void* grad_out, const void* x, const void* y, const void* sens, const float* mask,
+                                double* grad_eta, const gleam_dims* dims);
+GLEAM_API int gleam_dc_grad_y(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_y,
+                              const gleam_dims* dims);
+GLEAM_API int gleam_dc_grad_workspace_size(const gleam_dims* dims, uint64_t* bytes);
+
 /* ---- MoDL data-consistency step (Eq. 7, second line) -------------------------------------------
  *
  *     out = (A^H A + mu I)^{-1} (A^H y + mu z)
@@ -228,7 +283,8 @@ enum {
     GLEAM_K_COL_FWD = 7,
     GLEAM_K_COL_INV = 8,
     GLEAM_K_CG_VEC = 9,       /* image-sized vector kernels of the conjugate-gradient solve */
-    GLEAM_K_CLASSES = 10
+    GLEAM_K_FUSED3D = 10,     /* persistent kernel of the separable 3-D path (all three passes) */
+    GLEAM_K_CLASSES = 11
 };
 GLEAM_API uint64_t gleam_dc_launch_count(void);
 GLEAM_API int gleam_dc_profile_begin(void);

@@ -32,10 +32,12 @@ EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam
            "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end",
            "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes",
            "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size",
-           "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_adjoint"]
+           "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_adjoint",
+           "gleam_dc_check_status", "gleam_dc_debug_fused", "gleam_dc_fused_wait_stats", "gleam_dc_set_fused",
+           "gleam_dc_grad_eta", "gleam_dc_grad_y", "gleam_dc_grad_workspace_size"]
 
 KERNEL_CLASSES = ["zmap", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
-                  "col_inv", "cg_vec"]
+                  "col_inv", "cg_vec", "fused3d"]
 
 
 class gleam_dims(ctypes.Structure):
@@ -109,6 +111,20 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_modl_cg_vjp.restype = i32
         lib.gleam_modl_cg_workspace_size.argtypes = [dp, ctypes.POINTER(u64)]
         lib.gleam_modl_cg_workspace_size.restype = i32
+        lib.gleam_dc_check_status.argtypes = [dp]
+        lib.gleam_dc_check_status.restype = i32
+        lib.gleam_dc_fused_wait_stats.argtypes = [dp, ctypes.POINTER(u64), ctypes.c_int32]
+        lib.gleam_dc_fused_wait_stats.restype = i32
+        lib.gleam_dc_grad_eta.argtypes = [vp, vp, vp, vp, vp, vp, dp]
+        lib.gleam_dc_grad_eta.restype = i32
+        lib.gleam_dc_grad_y.argtypes = [vp, vp, vp, f32, vp, dp]
+        lib.gleam_dc_grad_y.restype = i32
+        lib.gleam_dc_grad_workspace_size.argtypes = [dp, ctypes.POINTER(u64)]
+        lib.gleam_dc_grad_workspace_size.restype = i32
+        lib.gleam_dc_set_fused.argtypes = [ctypes.c_int32]
+        lib.gleam_dc_set_fused.restype = None
+        lib.gleam_dc_debug_fused.argtypes = [ctypes.c_int32, u64]
+        lib.gleam_dc_debug_fused.restype = None
         lib.gleam_dc_launch_count.argtypes = []
         lib.gleam_dc_launch_count.restype = u64
         lib.gleam_dc_profile_begin.argtypes = []
@@ -197,6 +213,51 @@ def gleam_dc_forward_prepared(x, y, sens, mask, eta, out, dims: gleam_dims) -> N
     """gleam_dc_forward with the tables of an earlier gleam_dc_prepare(y, mask, dims)."""
     _check(load_library().gleam_dc_forward_prepared(_addr(x), _addr(y), _addr(sens), _addr(mask), float(eta),
                                                      _addr(out), ctypes.byref(dims)))
+
+
+def gleam_dc_check_status(dims: gleam_dims) -> int:
+    """Synchronises dims.stream and returns the device-side status of the work enqueued with these
+    dims and workspace: GLEAM_OK or GLEAM_ERR_TIMEOUT (a bounded wait between blocks ran out)."""
+    return int(load_library().gleam_dc_check_status(ctypes.byref(dims)))
+
+
+FUSED_WAIT_KINDS = ["ring_slot", "first_pass_done", "middle_pass_done", "sens_tile", "workspace_tile"]
+
+
+def gleam_dc_fused_wait_stats(dims: gleam_dims) -> dict:
+    """{kind: (microseconds summed over all blocks, waits that had to spin)} of the last persistent-kernel call."""
+    n = len(FUSED_WAIT_KINDS)
+    buf = (ctypes.c_uint64 * (2 * n))()
+    _check(load_library().gleam_dc_fused_wait_stats(ctypes.byref(dims), buf, n))
+    return {FUSED_WAIT_KINDS[i]: (buf[2 * i] * 1e-3, int(buf[2 * i + 1])) for i in range(n)}
+
+
+def gleam_dc_grad_workspace_size(dims: gleam_dims) -> int:
+    out = ctypes.c_uint64(0)
+    _check(load_library().gleam_dc_grad_workspace_size(ctypes.byref(dims), ctypes.byref(out)))
+    return int(out.value)
+
+
+def gleam_dc_grad_eta(grad_out, x, y, sens, mask, grad_eta, dims: gleam_dims) -> None:
+    """grad_eta[b] = -Re<g_b, A^H(A x - y)_b> (device float64, one value per batch example)."""
+    _check(load_library().gleam_dc_grad_eta(_addr(grad_out), _addr(x), _addr(y), _addr(sens), _addr(mask),
+                                             _addr(grad_eta), ctypes.byref(dims)))
+
+
+def gleam_dc_grad_y(grad_out, sens, mask, eta, grad_y, dims: gleam_dims) -> None:
+    """grad_y = eta Omega F S grad_out (complex64, layout of y)."""
+    _check(load_library().gleam_dc_grad_y(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_y),
+                                           ctypes.byref(dims)))
+
+
+def gleam_dc_set_fused(on: bool) -> None:
+    """Selects the persistent kernel of the separable 3-D path (off by default); call before sizing workspaces."""
+    load_library().gleam_dc_set_fused(1 if on else 0)
+
+
+def gleam_dc_debug_fused(withhold_item: int = -1, wait_limit_ns: int = 0) -> None:
+    """Test aid: withhold one item of the persistent 3-D kernel and / or shorten its wait limit."""
+    load_library().gleam_dc_debug_fused(int(withhold_item), int(wait_limit_ns))
 
 
 def gleam_dc_host_arena_size(dims: gleam_dims) -> int:

@@ -19,7 +19,7 @@
 namespace gleam {
 
 enum RowMode { ROW_FUSED = 0, ROW_FWD = 1, ROW_INV = 2 };
-enum ColMode { COL_Z = 0, COL_MID_SEP = 1, COL_MID_FULL = 2, COL_FWD = 3, COL_INV = 4 };
+enum ColMode { COL_Z = 0, COL_MID_SEP = 1, COL_MID_FULL = 2, COL_FWD = 3, COL_INV = 4, COL_GRADY = 5 };
 
 struct RowArgs {
     const cf* x;        // image-domain input (B,T,n0,n1,n2)
@@ -57,6 +57,8 @@ struct ColArgs {
     int ztiles;         // COL_Z: blocks launched per outer index (they stride over the tiles of ranks)
     float scale;        // COL_Z: g_ro g_pe / sqrt(N_ro N_pe);  COL_MID_FULL: g / sqrt(Ntot)
     float scale2;       // COL_MID_FULL: 1 / Ntot;  COL_MID_SEP: 1 / (n1 n2)
+    cf* ky_out;         // COL_GRADY: k-space output (B,C,T,V), written at the centred positions
+    int mask_pe;        // COL_GRADY: 0 = full mask (B,T,V); else the mask is readout-invariant with this many entries per image
 };
 
 constexpr int COLZ_SELF_MAX = 1024;   // COL_Z ranks a mask row of at most this many positions by itself
@@ -402,6 +404,37 @@ col_kernel(const ColArgs a) {
                 }
             }
         }
+    }
+
+    if (MODE == COL_GRADY) {
+        // Last axis of the forward operator A = Omega F S (Eq. 1) on W (already transformed along the other
+        // axes): out[p] = scale (-1)^{|p|} M[p] Fraw(.)[k] at the centred position p = sh(k) of every axis;
+        // `scale` carries the caller's factor (eta for the gradient with respect to y), g and 1/sqrt(Ntot).
+        if (actL) {
+            const long long unit = o;
+            const int t = (int)(unit % a.T);
+            const int b = (int)(unit / ((long long)a.C * a.T));
+            const long long V = (long long)a.n0 * a.n1 * a.n2;
+            const long long bt = (long long)b * a.T + t;
+            cf* dst = a.ky_out + unit * V;
+#pragma unroll
+            for (int k = 0; k < RL; ++k) {
+                const int kk = d.jL + P::BFL * k;
+                long long ps; int par;
+                if (a.rank == 2) {
+                    const int s1 = shift_half(kk, a.n1), s2 = shift_half(i, a.n2);
+                    ps = (long long)s1 * a.n2 + s2; par = (s1 + s2) & 1;
+                } else {
+                    const int i1 = i / a.n2, i2 = i % a.n2;
+                    const int s0 = shift_half(kk, a.n0), s1 = shift_half(i1, a.n1), s2 = shift_half(i2, a.n2);
+                    ps = ((long long)s0 * a.n1 + s1) * a.n2 + s2; par = (s0 + s1 + s2) & 1;
+                }
+                const float mv = a.mask_pe ? a.mask[bt * a.mask_pe + ps % a.mask_pe] : a.mask[bt * V + ps];
+                const float f = (par ? -a.scale : a.scale) * mv;
+                dst[ps] = cscale(u[k], f);
+            }
+        }
+        return;
     }
 
     E::inverse(u, v, tw, d, smem);

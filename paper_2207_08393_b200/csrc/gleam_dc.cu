@@ -13,10 +13,13 @@
 #include "../../include/gleam.h"
 #include "size_ops.cuh"
 #include "dc_rowtile.cuh"
+#include "dc_fused3d.cuh"
+#include "dc_fused_entry.h"
 #include "dc_entry.h"
 
 #include <atomic>
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <mutex>
 #include <vector>
@@ -147,7 +150,37 @@ struct Layout {
     // workspace (byte offsets)
     uint64_t off_z, off_zidx, off_zlist, off_zcount, off_m2c, off_zstart, off_zchunk, off_W, total;
     int G;  // readout slabs per chunk (rank 3 separable)
+    // fused persistent kernel of the separable 3-D path: control words first (at offset 0, the same
+    // for forward and VJP calls, so that gleam_dc_check_status finds them), then the ring of R slabs
+    bool fused;
+    uint64_t off_ctrl, ctrl_bytes, off_ring;
+    int R, L2, L3;
 };
+
+// Ring size and lags of the fused kernel, in slabs.  The groups of an SM take about four steps per
+// item and one block per SM is resident, so about three periods of items are in flight: P2 follows
+// P1 by L2 = 2 periods, P3 by L3 = 4, and the ring holds R = 8 slabs (42 MB for 8 coils of 320 x 256,
+// inside the 126 MB L2).  GLEAM_FUSED_RING="R,L2,L3" overrides (tuning aid, read once).
+static void fused_ring(int* R, int* L2, int* L3) {
+    static int v[3] = {0, 0, 0};
+    if (v[0] == 0) {
+        int r = 8, l2 = 2, l3 = 4;
+        const char* e = getenv("GLEAM_FUSED_RING");
+        if (e) { int a = 0, b = 0, c = 0; if (sscanf(e, "%d,%d,%d", &a, &b, &c) == 3 && a > c && c >= b && b >= 1 && a <= 64) { r = a; l2 = b; l3 = c; } }
+        v[1] = l2; v[2] = l3; v[0] = r;
+    }
+    *R = v[0]; *L2 = v[1]; *L3 = v[2];
+}
+// The persistent kernel is opt-in: measured on knee3d it is slower than the three whole-volume passes
+// (1.90 ms against 1.77 ms per VJP call), so the default keeps those.  GLEAM_FUSED=1 in the environment
+// or gleam_dc_set_fused(1) selects it; the choice changes the workspace layout, so it is made before
+// gleam_dc_workspace_size.
+static std::atomic<int> g_fused_on{-1};
+static bool fused_enabled() {
+    int v = g_fused_on.load(std::memory_order_relaxed);
+    if (v < 0) { const char* e = getenv("GLEAM_FUSED"); v = (e && e[0] == '1') ? 1 : 0; g_fused_on.store(v); }
+    return v == 1;
+}
 
 // Target size of the 3-D chunk workspace.  A chunk of about 48 MB would stay inside L2 between the
 // three kernels of a chunk, but at their present speed the kernels are bound by instruction issue,
@@ -184,6 +217,18 @@ static int make_layout(const gleam_dims* d, bool with_y, Layout* L) {
     L->separable = d->mask_kind == GLEAM_MASK_READOUT_INVARIANT;
     uint64_t off = 0;
     L->off_z = L->off_zidx = L->off_zlist = L->off_zcount = L->off_m2c = L->off_zstart = L->off_zchunk = L->off_W = 0; L->G = 0;
+    L->fused = false; L->off_ctrl = L->ctrl_bytes = L->off_ring = 0; L->R = L->L2 = L->L3 = 0;
+    if (L->separable && L->rank == 3 && fused_enabled() && fused3d_supported(L->n1, L->n2) &&
+        L->images * L->n0 < (1ll << 24)) {
+        L->fused = true;
+        fused_ring(&L->R, &L->L2, &L->L3);
+        const long long nslabs = L->images * L->n0;
+        if (L->R > nslabs + L->L3) L->R = (int)(nslabs + L->L3);      // never more slots than slabs in flight
+        if (L->R <= L->L3) L->R = L->L3 + 1;
+        L->off_ctrl = off; L->ctrl_bytes = (uint64_t)(64 + 3 * nslabs) * sizeof(int);
+        off = align_up(off + L->ctrl_bytes, 256);
+        L->off_ring = off; off = align_up(off + (uint64_t)L->R * L->C * L->n1 * L->n2 * sizeof(cf), 256);
+    }
     if (L->separable) {
         const long long pe = (L->rank == 2) ? L->n2 : (long long)L->n1 * L->n2;
         if (with_y) {
@@ -366,6 +411,20 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             ra.dot_rows = dot_rows;
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
+            if (L.fused && !y) {
+                // one persistent kernel walks all slabs; its counters start from zero
+                FusedArgs fa{};
+                fa.x = (const cf*)x; fa.sens = (const cf*)sens; fa.out = (cf*)out; fa.W = (cf*)(ws + L.off_ring);
+                fa.mask = mask; fa.zin = z; fa.zidx = ca.zidx; fa.m2c = ca.m2c; fa.zstart = ca.zstart;
+                fa.ctrl = (int*)(ws + L.off_ctrl); fa.eta = eta; fa.scale2 = 1.0f / (float)pe;
+                fa.C = L.C; fa.T = L.T; fa.Ts = L.Ts; fa.n0 = L.n0; fa.nslabs = (int)(L.images * L.n0);
+                fa.R = L.R; fa.L2 = L.L2; fa.L3 = L.L3;
+                fa.withhold = fused3d_withhold(); fa.limit_ns = fused3d_limit_ns();
+                CK(cudaMemsetAsync(fa.ctrl, 0, L.ctrl_bytes, s));
+                LAUNCH(GLEAM_K_FUSED3D, fused3d_launch(L.n1, fa, s));
+                CK(prof_mark(-1, s));
+                return GLEAM_OK;
+            }
             cf* W = (cf*)(ws + L.off_W);
             const PairOps* pair = find_pair(L.n1, L.n2);
             for (int i0 = 0; i0 < L.n0; i0 += L.G) {
@@ -416,6 +475,56 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
     return GLEAM_OK;
 }
 
+
+// ---- gradients of Eq. 3 with respect to the measurements and the step size ----
+// <g, a> per batch example, double accumulation in a fixed order: block partial sums, then one block per example.
+#define GRAD_THREADS 256
+#define GRAD_MAX_BLOCKS 512
+__global__ void __launch_bounds__(GRAD_THREADS) grad_eta_partial_kernel(const cf* __restrict__ g, const cf* __restrict__ x,
+                                                                        const cf* __restrict__ t, long long ne,
+                                                                        double* __restrict__ part) {
+    // t = x - A^H(Ax - y)  (the step with eta = 1), so A^H(Ax - y) = x - t
+    __shared__ double sh[GRAD_THREADS];
+    const long long base = (long long)blockIdx.y * ne;
+    double acc = 0.0;
+    for (long long i = (long long)blockIdx.x * GRAD_THREADS + threadIdx.x; i < ne; i += (long long)gridDim.x * GRAD_THREADS) {
+        const cf gv = g[base + i], xv = x[base + i], tv = t[base + i];
+        acc += (double)gv.x * ((double)xv.x - (double)tv.x) + (double)gv.y * ((double)xv.y - (double)tv.y);
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int o = GRAD_THREADS / 2; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) part[(long long)blockIdx.y * gridDim.x + blockIdx.x] = sh[0];
+}
+__global__ void grad_eta_final_kernel(const double* __restrict__ part, int nblocks, double* __restrict__ grad_eta) {
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (int i = 0; i < nblocks; ++i) s += part[(long long)blockIdx.x * nblocks + i];
+        grad_eta[blockIdx.x] = -s;
+    }
+}
+
+struct GradLayout { uint64_t dc_bytes, off_t, off_part, off_W, total; long long ne; int nblocks; };
+static int grad_layout(const gleam_dims* d, GradLayout* G) {
+    Layout L;
+    int rc = make_layout(d, true, &L);
+    if (rc != GLEAM_OK) return rc;
+    G->dc_bytes = align_up(L.total, 256);
+    G->ne = (long long)L.T * L.V;
+    long long nb = (G->ne + GRAD_THREADS * 8 - 1) / (GRAD_THREADS * 8);
+    G->nblocks = (int)(nb < 1 ? 1 : (nb > GRAD_MAX_BLOCKS ? GRAD_MAX_BLOCKS : nb));
+    uint64_t off = G->dc_bytes;
+    G->off_t = off; off = align_up(off + (uint64_t)L.images * L.V * sizeof(cf), 256);
+    G->off_part = off; off = align_up(off + (uint64_t)L.B * G->nblocks * sizeof(double), 256);
+    const uint64_t wbytes = (uint64_t)L.units * L.V * sizeof(cf);          // coil-volume workspace of the measurement gradient
+    G->off_W = 0;
+    G->total = off > wbytes ? off : align_up(wbytes, 256);
+    return GLEAM_OK;
+}
+
 }  // namespace gleam
 
 extern "C" {
@@ -459,6 +568,142 @@ GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes) {
     int rc = gleam::make_layout(dims, true, &L);
     if (rc != GLEAM_OK) return rc;
     *bytes = L.total;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_check_status(const gleam_dims* dims) {
+    if (!dims) return GLEAM_ERR_NULL_POINTER;
+    gleam::Layout L;
+    int rc = gleam::make_layout(dims, true, &L);
+    if (rc != GLEAM_OK) return rc;
+    if (cudaStreamSynchronize((cudaStream_t)dims->stream) != cudaSuccess) return GLEAM_ERR_CUDA;
+    if (!L.fused) return GLEAM_OK;                  // no kernel of this problem class waits on another block
+    if (!dims->workspace) return GLEAM_ERR_NULL_POINTER;
+    if (dims->workspace_bytes < L.total) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    int word = 0;
+    if (cudaMemcpy(&word, (const char*)dims->workspace + L.off_ctrl + sizeof(int), sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return GLEAM_ERR_CUDA;
+    return word == 0 ? GLEAM_OK : GLEAM_ERR_TIMEOUT;
+}
+
+GLEAM_API int gleam_dc_fused_wait_stats(const gleam_dims* dims, uint64_t* ns_and_counts, int32_t n_kinds) {
+    if (!dims || !ns_and_counts) return GLEAM_ERR_NULL_POINTER;
+    gleam::Layout L;
+    int rc = gleam::make_layout(dims, true, &L);
+    if (rc != GLEAM_OK) return rc;
+    for (int i = 0; i < 2 * n_kinds; ++i) ns_and_counts[i] = 0;
+    if (!L.fused) return GLEAM_OK;
+    if (!dims->workspace || dims->workspace_bytes < L.total) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    if (cudaStreamSynchronize((cudaStream_t)dims->stream) != cudaSuccess) return GLEAM_ERR_CUDA;
+    uint64_t w[10];
+    if (cudaMemcpy(w, (const char*)dims->workspace + L.off_ctrl + 8 * sizeof(int), sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return GLEAM_ERR_CUDA;
+    for (int i = 0; i < 2 * (n_kinds < 5 ? n_kinds : 5); ++i) ns_and_counts[i] = w[i];
+    return GLEAM_OK;
+}
+
+GLEAM_API void gleam_dc_set_fused(int32_t on) { gleam::g_fused_on.store(on ? 1 : 0); }
+
+GLEAM_API void gleam_dc_debug_fused(int32_t withhold_item, uint64_t wait_limit_ns) {
+    gleam::fused3d_set_debug(withhold_item, wait_limit_ns);
+}
+
+GLEAM_API int gleam_dc_grad_workspace_size(const gleam_dims* dims, uint64_t* bytes) {
+    if (!dims || !bytes) return GLEAM_ERR_NULL_POINTER;
+    gleam::GradLayout G;
+    int rc = gleam::grad_layout(dims, &G);
+    if (rc != GLEAM_OK) return rc;
+    *bytes = G.total;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_grad_eta(const void* grad_out, const void* x, const void* y, const void* sens, const float* mask,
+                                double* grad_eta, const gleam_dims* dims) {
+    using namespace gleam;
+    if (!dims || !grad_out || !x || !y || !sens || !mask || !grad_eta) return GLEAM_ERR_NULL_POINTER;
+    GradLayout G;
+    int rc = grad_layout(dims, &G);
+    if (rc != GLEAM_OK) return rc;
+    if (!dims->workspace) return GLEAM_ERR_NULL_POINTER;
+    if (dims->workspace_bytes < G.total) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    if (((uintptr_t)grad_out & 15) != 0 || ((uintptr_t)grad_eta & 7) != 0 || ((uintptr_t)dims->workspace & 255) != 0) return GLEAM_ERR_BAD_DIMS;
+    if ((rc = check_device_ptr(grad_out)) != GLEAM_OK || (rc = check_device_ptr(grad_eta)) != GLEAM_OK) return rc;
+    char* ws = (char*)dims->workspace;
+    const uint64_t img_b = (uint64_t)dims->batch * G.ne * sizeof(cf);
+    if (overlaps(ws, G.total, grad_out, img_b) || overlaps(ws, G.total, grad_eta, (uint64_t)dims->batch * 8) ||
+        overlaps(grad_eta, (uint64_t)dims->batch * 8, grad_out, img_b) || overlaps(grad_eta, (uint64_t)dims->batch * 8, x, img_b))
+        return GLEAM_ERR_ALIAS;
+    gleam_dims d = *dims;
+    d.workspace = ws; d.workspace_bytes = G.dc_bytes;
+    cf* t = (cf*)(ws + G.off_t);
+    rc = run(x, y, sens, mask, 1.0f, t, &d, RUN_ALL, nullptr, true);       // every argument check before anything is enqueued
+    if (rc != GLEAM_OK) return rc;
+    rc = run(x, y, sens, mask, 1.0f, t, &d);                               // t = x - A^H (A x - y)
+    if (rc != GLEAM_OK) return rc;
+    cudaStream_t s = (cudaStream_t)dims->stream;
+    double* part = (double*)(ws + G.off_part);
+    if (prof_mark(GLEAM_K_CG_VEC, s) != cudaSuccess) return GLEAM_ERR_CUDA;
+    grad_eta_partial_kernel<<<dim3((unsigned)G.nblocks, (unsigned)dims->batch), GRAD_THREADS, 0, s>>>((const cf*)grad_out, (const cf*)x, t, G.ne, part);
+    if (cudaGetLastError() != cudaSuccess) return GLEAM_ERR_CUDA;
+    if (prof_mark(GLEAM_K_CG_VEC, s) != cudaSuccess) return GLEAM_ERR_CUDA;
+    grad_eta_final_kernel<<<(unsigned)dims->batch, 32, 0, s>>>(part, G.nblocks, grad_eta);
+    if (cudaGetLastError() != cudaSuccess) return GLEAM_ERR_CUDA;
+    if (prof_mark(-1, s) != cudaSuccess) return GLEAM_ERR_CUDA;
+    return GLEAM_OK;
+}
+
+GLEAM_API int gleam_dc_grad_y(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_y,
+                              const gleam_dims* dims) {
+    using namespace gleam;
+    if (!dims || !grad_out || !sens || !mask || !grad_y) return GLEAM_ERR_NULL_POINTER;
+    Layout L;
+    int rc = make_layout(dims, false, &L);
+    if (rc != GLEAM_OK) return rc;
+    GradLayout G;
+    if ((rc = grad_layout(dims, &G)) != GLEAM_OK) return rc;
+    if (!dims->workspace) return GLEAM_ERR_NULL_POINTER;
+    if (dims->workspace_bytes < G.total) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    if (((uintptr_t)dims->workspace & 255) != 0) return GLEAM_ERR_BAD_DIMS;
+    const void* ptrs[5] = {grad_out, sens, mask, grad_y, dims->workspace};
+    for (int i = 0; i < 5; ++i) {
+        if (((uintptr_t)ptrs[i] & 15) != 0) return GLEAM_ERR_BAD_DIMS;
+        if ((rc = check_device_ptr(ptrs[i])) != GLEAM_OK) return rc;
+    }
+    const uint64_t img_b = (uint64_t)L.images * L.V * sizeof(cf), ksp_b = (uint64_t)L.units * L.V * sizeof(cf);
+    const uint64_t sens_b = (uint64_t)L.B * L.C * L.Ts * L.V * sizeof(cf);
+    const long long pe = (L.rank == 2) ? L.n2 : (long long)L.n1 * L.n2;
+    const uint64_t mask_b = (uint64_t)L.images * (L.separable ? pe : L.V) * sizeof(float);
+    if (overlaps(grad_y, ksp_b, grad_out, img_b) || overlaps(grad_y, ksp_b, sens, sens_b) || overlaps(grad_y, ksp_b, mask, mask_b) ||
+        overlaps(dims->workspace, G.total, grad_y, ksp_b) || overlaps(dims->workspace, G.total, grad_out, img_b) ||
+        overlaps(dims->workspace, G.total, sens, sens_b) || overlaps(dims->workspace, G.total, mask, mask_b))
+        return GLEAM_ERR_ALIAS;
+    cudaStream_t s = (cudaStream_t)dims->stream;
+    cf* W = (cf*)((char*)dims->workspace + G.off_W);
+    const SizeOps* op2 = find_size(L.n2);
+    const SizeOps* op1 = find_size(L.n1);
+    const SizeOps* op0 = (L.rank == 3) ? find_size(L.n0) : nullptr;
+    RowArgs ra{};
+    ra.x = (const cf*)grad_out; ra.sens = (const cf*)sens; ra.W = W; ra.eta = 0.f;
+    ra.C = L.C; ra.T = L.T; ra.Ts = L.Ts; ra.RPB = L.n0 * L.n1; ra.rpb = ra.RPB; ra.row0 = 0; ra.nrows = L.images * ra.rpb;
+    LAUNCH(GLEAM_K_ROW_FWD, op2->row(ROW_FWD, ra, s));
+    ColArgs ca{};
+    ca.C = L.C; ca.T = L.T; ca.rank = L.rank; ca.n0 = L.n0; ca.n1 = L.n1; ca.n2 = L.n2; ca.W = W;
+    const float gs = gsign(L.n2) * gsign(L.n1) * (L.rank == 3 ? gsign(L.n0) : 1.f);
+    const double ntot = (L.rank == 3) ? (double)L.V : (double)L.n1 * L.n2;
+    ColArgs cy = ca;
+    cy.mask = mask; cy.ky_out = (cf*)grad_y; cy.mask_pe = L.separable ? (int)pe : 0;
+    cy.scale = eta * gs / (float)sqrt(ntot);
+    if (L.rank == 2) {
+        cy.es = L.n2; cy.nouter = L.units;
+        LAUNCH(GLEAM_K_COL_FWD, op1->col(COL_GRADY, cy, s));
+    } else {
+        ColArgs c1 = ca;
+        c1.es = L.n2; c1.nouter = L.units * L.n0;
+        LAUNCH(GLEAM_K_COL_FWD, op1->col(COL_FWD, c1, s));
+        cy.es = L.n1 * L.n2; cy.nouter = L.units;
+        LAUNCH(GLEAM_K_COL_FWD, op0->col(COL_GRADY, cy, s));
+    }
+    CK(prof_mark(-1, s));
     return GLEAM_OK;
 }
 

@@ -174,6 +174,7 @@ struct SizeImpl {
             case COL_MID_FULL: return launch_col<PC, LC, COL_MID_FULL>(a, s);
             case COL_FWD:      return launch_col<PC, LC, COL_FWD>(a, s);
             case COL_INV:      return launch_col<PC, LC, COL_INV>(a, s);
+            case COL_GRADY:    return launch_col<PC, LC, COL_GRADY>(a, s);
         }
         return cudaErrorInvalidValue;
     }

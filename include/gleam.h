@@ -217,6 +217,32 @@ GLEAM_API int gleam_dc_forward_prepared(const void* x, const void* y, const void
 GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mask, void* out,
                                const gleam_dims* dims);
 
+/* ---- bridge to the learned prior ---------------------------------------------------------------------
+ * The paper's networks take and return complex images as two real channels (real part, imaginary part;
+ * Implementation / Training) and are trained with an l1 loss on complex images.  The _layout variants of
+ * the two main calls read and / or write the image-side arrays directly in that form,
+ *     (B, 2, T, n0, n1, n2) float32, channel 0 = real part, channel 1 = imaginary part,
+ * inside the kernels that load x and store out, so no conversion pass is needed on either side of the
+ * prior.  layout: GLEAM_X_CHANNELS (x / grad_out is two-channel), GLEAM_OUT_CHANNELS (out / grad_in is);
+ * 0 gives gleam_dc_forward / gleam_dc_vjp.  In place (out == x) needs both or neither.  With a layout flag
+ * the opt-in persistent kernel is not used.
+ *
+ * gleam_l1_loss:  loss = mean over all B T n0 n1 n2 complex elements of |x - ref|  (device double), and, if
+ * grad is not null, grad = (x - ref) / |x - ref| / N, zero where x = ref: the gradient a real loss sends
+ * back through a complex tensor (conjugate-Wirtinger convention), in the layout GLEAM_OUT_CHANNELS selects.
+ * ref is complex64 (B, T, n0, n1, n2); x in the layout GLEAM_X_CHANNELS selects.  The mean is accumulated in
+ * double precision in a fixed order.  dims->workspace: gleam_l1_loss_workspace_size() bytes.
+ */
+#define GLEAM_X_CHANNELS 1u
+#define GLEAM_OUT_CHANNELS 2u
+GLEAM_API int gleam_dc_forward_layout(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                      void* out, const gleam_dims* dims, uint32_t layout);
+GLEAM_API int gleam_dc_vjp_layout(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
+                                  const gleam_dims* dims, uint32_t layout);
+GLEAM_API int gleam_l1_loss(const void* x, const void* ref, double* loss, void* grad, const gleam_dims* dims,
+                            uint32_t layout);
+GLEAM_API uint64_t gleam_l1_loss_workspace_size(void);
+
 /* ---- gradients of Eq. 3 with respect to the step size and the measurements --------------------------
  * out = x - eta A^H (A x - y) is linear in eta and affine in y.  For a cotangent g = grad_out of the
  * output (conjugate-Wirtinger convention, as for gleam_dc_vjp):

@@ -24,6 +24,9 @@ GLEAM_ERR_CUDA = -7
 GLEAM_ERR_UNIMPLEMENTED = -8
 GLEAM_ERR_TIMEOUT = -9
 
+GLEAM_X_CHANNELS = 1
+GLEAM_OUT_CHANNELS = 2
+
 GLEAM_MASK_FULL = 0
 GLEAM_MASK_READOUT_INVARIANT = 1
 
@@ -34,7 +37,8 @@ EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam
            "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size",
            "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_adjoint",
            "gleam_dc_check_status", "gleam_dc_debug_fused", "gleam_dc_fused_wait_stats", "gleam_dc_set_fused",
-           "gleam_dc_grad_eta", "gleam_dc_grad_y", "gleam_dc_grad_workspace_size"]
+           "gleam_dc_grad_eta", "gleam_dc_grad_y", "gleam_dc_grad_workspace_size",
+           "gleam_dc_forward_layout", "gleam_dc_vjp_layout", "gleam_l1_loss", "gleam_l1_loss_workspace_size"]
 
 KERNEL_CLASSES = ["zmap", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
                   "col_inv", "cg_vec", "fused3d"]
@@ -121,6 +125,15 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_dc_grad_y.restype = i32
         lib.gleam_dc_grad_workspace_size.argtypes = [dp, ctypes.POINTER(u64)]
         lib.gleam_dc_grad_workspace_size.restype = i32
+        u32 = ctypes.c_uint32
+        lib.gleam_dc_forward_layout.argtypes = [vp, vp, vp, vp, f32, vp, dp, u32]
+        lib.gleam_dc_forward_layout.restype = i32
+        lib.gleam_dc_vjp_layout.argtypes = [vp, vp, vp, f32, vp, dp, u32]
+        lib.gleam_dc_vjp_layout.restype = i32
+        lib.gleam_l1_loss.argtypes = [vp, vp, vp, vp, dp, u32]
+        lib.gleam_l1_loss.restype = i32
+        lib.gleam_l1_loss_workspace_size.argtypes = []
+        lib.gleam_l1_loss_workspace_size.restype = u64
         lib.gleam_dc_set_fused.argtypes = [ctypes.c_int32]
         lib.gleam_dc_set_fused.restype = None
         lib.gleam_dc_debug_fused.argtypes = [ctypes.c_int32, u64]
@@ -248,6 +261,26 @@ def gleam_dc_grad_y(grad_out, sens, mask, eta, grad_y, dims: gleam_dims) -> None
     """grad_y = eta Omega F S grad_out (complex64, layout of y)."""
     _check(load_library().gleam_dc_grad_y(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_y),
                                            ctypes.byref(dims)))
+
+
+def gleam_dc_forward_layout(x, y, sens, mask, eta, out, dims: gleam_dims, layout: int) -> None:
+    """gleam_dc_forward with x and / or out in the two-real-channel layout (B, 2, T, n0, n1, n2) float32."""
+    _check(load_library().gleam_dc_forward_layout(_addr(x), _addr(y), _addr(sens), _addr(mask), float(eta), _addr(out),
+                                                   ctypes.byref(dims), int(layout)))
+
+
+def gleam_dc_vjp_layout(grad_out, sens, mask, eta, grad_in, dims: gleam_dims, layout: int) -> None:
+    _check(load_library().gleam_dc_vjp_layout(_addr(grad_out), _addr(sens), _addr(mask), float(eta), _addr(grad_in),
+                                               ctypes.byref(dims), int(layout)))
+
+
+def gleam_l1_loss_workspace_size() -> int:
+    return int(load_library().gleam_l1_loss_workspace_size())
+
+
+def gleam_l1_loss(x, ref, loss, grad, dims: gleam_dims, layout: int = 0) -> None:
+    """loss (device float64 scalar) = mean |x - ref|; grad (optional) = (x - ref)/|x - ref|/N."""
+    _check(load_library().gleam_l1_loss(_addr(x), _addr(ref), _addr(loss), _addr(grad), ctypes.byref(dims), int(layout)))
 
 
 def gleam_dc_set_fused(on: bool) -> None:

@@ -13,7 +13,8 @@ enum { RUN_ALL = 0, RUN_PREPARE = 1, RUN_APPLY = 2 };
 // enqueues on d->stream, returns GLEAM_OK or a GLEAM_ERR_* code.  check_only: the argument checks
 // alone (callers that must enqueue something of their own before the step run them first).
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode = RUN_ALL, double* dot_rows = nullptr, bool check_only = false);
+        const gleam_dims* d, int mode = RUN_ALL, double* dot_rows = nullptr, bool check_only = false,
+        int layout = 0);     // layout: GLEAM_X_CHANNELS | GLEAM_OUT_CHANNELS (two-real-channel image arrays)
 
 // dot_rows (device, one double per image row, B*T*n1): the one-pass 2-D kernel also stores
 // Re<x_row, out_row> of every row it writes, so that a caller's inner product <x, out> needs no

@@ -36,7 +36,24 @@ struct RowArgs {
     int RPB;            // rows of a full image (n0*n1)
     long long nrows;    // B*T*rpb
     double* dot_rows;   // ROW_FUSED (warp-resident form): if not null, Re<x, out> of every image row, (B*T*rpb)
+    // Two-real-channel layout (B, 2, T, n0, n1, n2) float32 of the image-side arrays (the form the learned
+    // prior takes and returns): real index of complex element e of example b = e + b * plane, the imaginary
+    // part `plane` further on (plane = T * n0 * n1 * n2).
+    int x_planar, out_planar;
+    long long plane;
 };
+
+// image-side element e (complex-element offset in the (B,T,V) array) of example b, in either layout
+__device__ __forceinline__ cf load_image(const cf* x, long long e, int planar, int b, long long plane) {
+    if (!planar) return x[e];
+    const float* xf = reinterpret_cast<const float*>(x) + e + (long long)b * plane;
+    return make_float2(xf[0], xf[plane]);
+}
+__device__ __forceinline__ void store_image(cf* out, long long e, cf v, int planar, int b, long long plane) {
+    if (!planar) { out[e] = v; return; }
+    float* of = reinterpret_cast<float*>(out) + e + (long long)b * plane;
+    of[0] = v.x; of[plane] = v.y;
+}
 
 struct ColArgs {
     cf* W;              // in-place data (COL_MID_*, COL_FWD, COL_INV)
@@ -100,7 +117,7 @@ row_kernel(const RowArgs a) {
     if (MODE != ROW_INV) {
         if (act0) {
 #pragma unroll
-            for (int m = 0; m < R0; ++m) xv[m] = a.x[x_off + d.j0 + P::BF0 * m];
+            for (int m = 0; m < R0; ++m) xv[m] = load_image(a.x, x_off + d.j0 + P::BF0 * m, a.x_planar, b0, a.plane);
         }
     }
     float m2v[RL];
@@ -209,12 +226,12 @@ row_kernel(const RowArgs a) {
         if (act0) {
             if (MODE == ROW_INV) {
 #pragma unroll
-                for (int m = 0; m < R0; ++m) xv[m] = a.x[x_off + d.j0 + P::BF0 * m];
+                for (int m = 0; m < R0; ++m) xv[m] = load_image(a.x, x_off + d.j0 + P::BF0 * m, a.x_planar, b0, a.plane);
             }
 #pragma unroll
             for (int m = 0; m < R0; ++m)
-                a.out[x_off + d.j0 + P::BF0 * m] =
-                    make_float2(fmaf(-a.eta, acc[m].x, xv[m].x), fmaf(-a.eta, acc[m].y, xv[m].y));
+                store_image(a.out, x_off + d.j0 + P::BF0 * m,
+                            make_float2(fmaf(-a.eta, acc[m].x, xv[m].x), fmaf(-a.eta, acc[m].y, xv[m].y)), a.out_planar, b0, a.plane);
         }
     }
 }

@@ -28,6 +28,7 @@ struct TileArgs {
     float eta, scale2;
     int C, T, Ts, n0, G, i0_start;
     long long nunits;                         // B*C*T
+    int x_planar, out_planar; long long plane; // two-real-channel layout of x / out (see RowArgs)
 };
 
 template <class PZ, int RY, int BY>
@@ -105,7 +106,7 @@ rowtile_kernel(const TileArgs a) {
     cf xreg[R0], acc[R0];
     if (a0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) { xreg[m] = a.x[x_off + jz + PZ::BF0 * m]; acc[m] = make_float2(0.f, 0.f); }
+        for (int m = 0; m < R0; ++m) { xreg[m] = load_image(a.x, x_off + jz + PZ::BF0 * m, a.x_planar, b, a.plane); acc[m] = make_float2(0.f, 0.f); }
     }
     issue_s(0);
     // pass 3: the column values of the first coil (one kz column per thread; THREADS >= NZ is not
@@ -211,7 +212,7 @@ rowtile_kernel(const TileArgs a) {
     if (INV && a0) {
 #pragma unroll
         for (int m = 0; m < R0; ++m)
-            a.out[x_off + jz + PZ::BF0 * m] = make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y));
+            store_image(a.out, x_off + jz + PZ::BF0 * m, make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y)), a.out_planar, b, a.plane);
     }
 }
 

@@ -133,7 +133,15 @@ warpline_kernel(const RowArgs a) {
             const long long bto = __shfl_sync(0xffffffffu, (long long)bt, ll * TPL);
             if (!ok) continue;
             if (WL::HAS_X) {
-                for (int i = lane; i < N / 2; i += 32) cp_async16(sX + ll * N + 2 * i, a.x + xo + 2 * i);
+                if (!a.x_planar) {
+                    for (int i = lane; i < N / 2; i += 32) cp_async16(sX + ll * N + 2 * i, a.x + xo + 2 * i);
+                } else {
+                    // two-channel layout: the line's real parts, then its imaginary parts, land interleaved
+                    const long long bo = __shfl_sync(0xffffffffu, (long long)b, ll * TPL);
+                    const float* xf = reinterpret_cast<const float*>(a.x) + xo + bo * a.plane;
+                    float* dst = reinterpret_cast<float*>(sX + ll * N);
+                    for (int i = lane; i < N; i += 32) { dst[2 * i] = xf[i]; dst[2 * i + 1] = xf[a.plane + i]; }
+                }
             }
             if (MODE == ROW_FUSED) {
                 // scaled mask^2 in raw k order and, with z, the rank of every sampled k (the order
@@ -159,7 +167,7 @@ warpline_kernel(const RowArgs a) {
         cf xreg[R0];     // ROW_FWD / ROW_INV: x fetched once per group and held in registers
         if (!WL::HAS_X && a0 && row_ok) {
 #pragma unroll
-            for (int m = 0; m < R0; ++m) xreg[m] = a.x[x_off + j + P::BF0 * m];
+            for (int m = 0; m < R0; ++m) xreg[m] = load_image(a.x, x_off + j + P::BF0 * m, a.x_planar, b, a.plane);
         }
 #pragma unroll
         for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
@@ -278,7 +286,7 @@ warpline_kernel(const RowArgs a) {
                 for (int m = 0; m < R0; ++m) {
                     const cf xv = WL::HAS_X ? sX[l * N + j + P::BF0 * m] : xreg[m];
                     const cf ov = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
-                    a.out[x_off + j + P::BF0 * m] = ov;
+                    store_image(a.out, x_off + j + P::BF0 * m, ov, a.out_planar, b, a.plane);
                     if (MODE == ROW_FUSED && a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;
                 }
             }

@@ -311,7 +311,7 @@ bool dot_rows_supported(const gleam_dims* d) {
 }
 
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode, double* dot_rows, bool check_only) {
+        const gleam_dims* d, int mode, double* dot_rows, bool check_only, int layout) {
     if (!d || !mask) return GLEAM_ERR_NULL_POINTER;
     if (mode == RUN_PREPARE) {
         if (!y) return GLEAM_ERR_NULL_POINTER;
@@ -341,8 +341,10 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         if (rc != GLEAM_OK) return rc;
     }
     // aliasing: out may equal x exactly; nothing else may overlap an output or the workspace
+    if (layout & ~(GLEAM_X_CHANNELS | GLEAM_OUT_CHANNELS)) return GLEAM_ERR_BAD_DIMS;
     if (mode != RUN_PREPARE) {
         if (out != x && overlaps(out, img_b, x, img_b)) return GLEAM_ERR_ALIAS;
+        if (out == x && ((layout & GLEAM_X_CHANNELS) != 0) != ((layout & GLEAM_OUT_CHANNELS) != 0)) return GLEAM_ERR_ALIAS;
         if (overlaps(out, img_b, sens, sens_b) || overlaps(out, img_b, mask, mask_b)) return GLEAM_ERR_ALIAS;
         if (y && overlaps(out, img_b, y, ksp_b)) return GLEAM_ERR_ALIAS;
     }
@@ -364,6 +366,8 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
     RowArgs ra{};
     ra.x = (const cf*)x; ra.sens = (const cf*)sens; ra.out = (cf*)out; ra.eta = eta;
     ra.C = L.C; ra.T = L.T; ra.Ts = L.Ts; ra.RPB = L.n0 * L.n1;
+    ra.x_planar = (layout & GLEAM_X_CHANNELS) ? 1 : 0; ra.out_planar = (layout & GLEAM_OUT_CHANNELS) ? 1 : 0;
+    ra.plane = (long long)L.T * L.V;
     ColArgs ca{};
     ca.C = L.C; ca.T = L.T; ca.rank = L.rank; ca.n0 = L.n0; ca.n1 = L.n1; ca.n2 = L.n2;
 
@@ -411,7 +415,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             ra.dot_rows = dot_rows;
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
-            if (L.fused && !y) {
+            if (L.fused && !y && layout == 0) {
                 // one persistent kernel walks all slabs; its counters start from zero
                 FusedArgs fa{};
                 fa.x = (const cf*)x; fa.sens = (const cf*)sens; fa.out = (cf*)out; fa.W = (cf*)(ws + L.off_ring);
@@ -435,6 +439,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
                     ta.x = (const cf*)x; ta.sens = (const cf*)sens; ta.out = (cf*)out; ta.V = W; ta.mask = mask;
                     ta.zin = z; ta.zidx = ca.zidx; ta.m2c = ca.m2c; ta.zstart = ca.zstart; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
                     ta.C = L.C; ta.T = L.T; ta.Ts = L.Ts; ta.n0 = L.n0; ta.G = g; ta.i0_start = i0; ta.nunits = L.units;
+                    ta.x_planar = ra.x_planar; ta.out_planar = ra.out_planar; ta.plane = ra.plane;
                     LAUNCH(GLEAM_K_ROW_FWD, pair->fwd(ta, L.images, s));
                     LAUNCH(GLEAM_K_COL_MID_SEP, pair->mid(ta, s));
                     LAUNCH(GLEAM_K_ROW_INV, pair->inv(ta, L.images, s));
@@ -507,6 +512,43 @@ __global__ void grad_eta_final_kernel(const double* __restrict__ part, int nbloc
     }
 }
 
+
+// ---- complex l1 loss between an image and a reference (training loss of the paper's networks) ----
+// loss = mean |x - r|; grad = (x - r) / |x - r| / N (zero where x = r).  Block partial sums in double, summed
+// by one thread in block order: deterministic.
+__global__ void __launch_bounds__(GRAD_THREADS) l1_partial_kernel(const cf* __restrict__ x, const cf* __restrict__ r, cf* __restrict__ grad,
+                                                                  long long ne, int B, int x_planar, int g_planar, long long plane,
+                                                                  float inv_n, double* __restrict__ part) {
+    __shared__ double sh[GRAD_THREADS];
+    double acc = 0.0;
+    const long long n = ne * B;
+    for (long long i = (long long)blockIdx.x * GRAD_THREADS + threadIdx.x; i < n; i += (long long)gridDim.x * GRAD_THREADS) {
+        const int b = (int)(i / ne);
+        const cf xv = load_image(x, i, x_planar, b, plane), rv = r[i];
+        const float dx = xv.x - rv.x, dy = xv.y - rv.y;
+        const float m = sqrtf(dx * dx + dy * dy);
+        acc += (double)m;
+        if (grad) {
+            const float s = m > 0.f ? inv_n / m : 0.f;
+            store_image(grad, i, make_float2(dx * s, dy * s), g_planar, b, plane);
+        }
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int o = GRAD_THREADS / 2; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) part[blockIdx.x] = sh[0];
+}
+__global__ void l1_final_kernel(const double* __restrict__ part, int nblocks, double inv_n, double* __restrict__ loss) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double s = 0.0;
+        for (int i = 0; i < nblocks; ++i) s += part[i];
+        *loss = s * inv_n;
+    }
+}
+
 struct GradLayout { uint64_t dc_bytes, off_t, off_part, off_W, total; long long ne; int nblocks; };
 static int grad_layout(const gleam_dims* d, GradLayout* G) {
     Layout L;
@@ -538,6 +580,17 @@ GLEAM_API int gleam_dc_forward(const void* x, const void* y, const void* sens, c
 GLEAM_API int gleam_dc_vjp(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
                  const gleam_dims* dims) {
     return gleam::run(grad_out, nullptr, sens, mask, eta, grad_in, dims);
+}
+
+GLEAM_API int gleam_dc_forward_layout(const void* x, const void* y, const void* sens, const float* mask, float eta,
+                                      void* out, const gleam_dims* dims, uint32_t layout) {
+    if (!y) return GLEAM_ERR_NULL_POINTER;
+    return gleam::run(x, y, sens, mask, eta, out, dims, gleam::RUN_ALL, nullptr, false, (int)layout);
+}
+
+GLEAM_API int gleam_dc_vjp_layout(const void* grad_out, const void* sens, const float* mask, float eta, void* grad_in,
+                                  const gleam_dims* dims, uint32_t layout) {
+    return gleam::run(grad_out, nullptr, sens, mask, eta, grad_in, dims, gleam::RUN_ALL, nullptr, false, (int)layout);
 }
 
 GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mask, void* out, const gleam_dims* dims) {
@@ -606,6 +659,43 @@ GLEAM_API void gleam_dc_set_fused(int32_t on) { gleam::g_fused_on.store(on ? 1 :
 
 GLEAM_API void gleam_dc_debug_fused(int32_t withhold_item, uint64_t wait_limit_ns) {
     gleam::fused3d_set_debug(withhold_item, wait_limit_ns);
+}
+
+GLEAM_API uint64_t gleam_l1_loss_workspace_size(void) { return GRAD_MAX_BLOCKS * sizeof(double); }
+
+GLEAM_API int gleam_l1_loss(const void* x, const void* ref, double* loss, void* grad, const gleam_dims* dims, uint32_t layout) {
+    using namespace gleam;
+    if (!dims || !x || !ref || !loss) return GLEAM_ERR_NULL_POINTER;
+    Layout L;
+    int rc = make_layout(dims, false, &L);
+    if (rc != GLEAM_OK) return rc;
+    if (layout & ~(GLEAM_X_CHANNELS | GLEAM_OUT_CHANNELS)) return GLEAM_ERR_BAD_DIMS;
+    if (!dims->workspace) return GLEAM_ERR_NULL_POINTER;
+    if (dims->workspace_bytes < gleam_l1_loss_workspace_size()) return GLEAM_ERR_WORKSPACE_TOO_SMALL;
+    if (((uintptr_t)x & 7) || ((uintptr_t)ref & 7) || ((uintptr_t)loss & 7) || ((uintptr_t)grad & 7) || ((uintptr_t)dims->workspace & 255)) return GLEAM_ERR_BAD_DIMS;
+    const void* ptrs[5] = {x, ref, loss, grad, dims->workspace};
+    for (int i = 0; i < 5; ++i) if (ptrs[i] && (rc = check_device_ptr(ptrs[i])) != GLEAM_OK) return rc;
+    const uint64_t img_b = (uint64_t)L.images * L.V * sizeof(cf);
+    if (grad && grad != x && (overlaps(grad, img_b, x, img_b) || overlaps(grad, img_b, ref, img_b))) return GLEAM_ERR_ALIAS;
+    if (grad == x && ((layout & GLEAM_X_CHANNELS) != 0) != ((layout & GLEAM_OUT_CHANNELS) != 0)) return GLEAM_ERR_ALIAS;
+    if (overlaps(dims->workspace, gleam_l1_loss_workspace_size(), x, img_b) || overlaps(dims->workspace, gleam_l1_loss_workspace_size(), ref, img_b) ||
+        (grad && overlaps(dims->workspace, gleam_l1_loss_workspace_size(), grad, img_b)) || overlaps(loss, 8, x, img_b) ||
+        (grad && overlaps(loss, 8, grad, img_b)))
+        return GLEAM_ERR_ALIAS;
+    const long long ne = (long long)L.T * L.V, n = ne * L.B;
+    long long nb = (n + GRAD_THREADS * 8 - 1) / (GRAD_THREADS * 8);
+    const int nblocks = (int)(nb < 1 ? 1 : (nb > GRAD_MAX_BLOCKS ? GRAD_MAX_BLOCKS : nb));
+    cudaStream_t s = (cudaStream_t)dims->stream;
+    double* part = (double*)dims->workspace;
+    CK(prof_mark(GLEAM_K_CG_VEC, s));
+    l1_partial_kernel<<<nblocks, GRAD_THREADS, 0, s>>>((const cf*)x, (const cf*)ref, (cf*)grad, ne, L.B, (layout & GLEAM_X_CHANNELS) ? 1 : 0,
+                                                       (layout & GLEAM_OUT_CHANNELS) ? 1 : 0, ne, (float)(1.0 / (double)n), part);
+    CK(cudaGetLastError());
+    CK(prof_mark(GLEAM_K_CG_VEC, s));
+    l1_final_kernel<<<1, 32, 0, s>>>(part, nblocks, 1.0 / (double)n, loss);
+    CK(cudaGetLastError());
+    CK(prof_mark(-1, s));
+    return GLEAM_OK;
 }
 
 GLEAM_API int gleam_dc_grad_workspace_size(const gleam_dims* dims, uint64_t* bytes) {

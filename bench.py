@@ -380,6 +380,29 @@ def run_ours(args, w):
         split[0] += ef[0].elapsed_time(ef[1]) / prof_steps / chain      # per call
         split[1] += ef[1].elapsed_time(ef[2]) / prof_steps / chain
 
+    # ---- cost of reading and writing the image in the prior's two-real-channel layout inside the kernels ----
+    g_ch = torch.stack([tg.real, tg.imag], dim=1).contiguous()
+    gin_ch = [torch.empty_like(g_ch), torch.empty_like(g_ch)]
+    both = g.GLEAM_X_CHANNELS | g.GLEAM_OUT_CHANNELS
+
+    def vjp_chain_channels():
+        src = g_ch
+        for i in range(chain):
+            g.gleam_dc_vjp_layout(src, ts, tm, w.eta, gin_ch[i % 2], dc.dims(), both)
+            src = gin_ch[i % 2]
+
+    lay = [0.0, 0.0]
+    for _ in range(prof_steps):
+        for k, fn in enumerate((vjp_chain, vjp_chain_channels)):
+            if flush is not None:
+                flush.fill_(1)
+            ef[0].record(stream); fn()
+            ef[1].record(stream); torch.cuda.synchronize()
+            lay[k] += ef[0].elapsed_time(ef[1]) / prof_steps / chain
+    layout_cost = {"vjp_us_complex64": lay[0] * 1e3, "vjp_us_two_channel_in_and_out": lay[1] * 1e3,
+                   "relative_cost": lay[1] / lay[0] - 1.0}
+    del g_ch, gin_ch
+
     # ---- the same chain with the y-dependent tables computed once per step (gleam_dc_prepare) ----
     prepared = None
     if chain > 1 and not full_mask:
@@ -514,6 +537,7 @@ def run_ours(args, w):
         "call_roofline": ns,
         "prepared_chain": prepared,
         "warm_l2": warm,
+        "two_channel_layout": layout_cost,
         "kernels": kernels,
         "cpu_baseline": cpu,
     }

@@ -183,7 +183,12 @@ GLEAM_API int gleam_dc_host_arena_size(const gleam_dims* dims, uint64_t* bytes);
  *     GLEAM_ERR_WORKSPACE_TOO_SMALL and launch nothing.
  *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *   - The first call on each device looks up the array's device address (once, with that device
- *     current); make that first call before any stream capture begins.
+ *     current); make that first call before any stream capture begins.  With CUDA's lazy module
+ *     loading the array itself comes into being when the library's device code is first loaded on a
+ *     device, which may be that first call (or any earlier call of this library there): that one
+ *     call can then take device memory and synchronise implicitly, and fails with GLEAM_ERR_CUDA if
+ *     64 MiB are no longer free.  Make it at start-up, before the device's memory is handed out;
+ *     every later call leaves the amount of free device memory unchanged.
  *   - All calls share the one array, which keeps whatever the previous call left in it; the
  *     kernels write every scratch element before reading it, so no clearing is needed.  Two calls
  *     whose GPU work overlaps (different streams, or different host threads on one device) race on

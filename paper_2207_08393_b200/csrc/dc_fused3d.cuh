@@ -18,10 +18,16 @@
 // the limit the block raises the error word, stops starting work, and the host reports
 // GLEAM_ERR_TIMEOUT from gleam_dc_check_status.
 //
-// Block = 17 warps: two compute groups of 256 threads that take half of the coils of an item each
-// (the coil sum of P3 is completed through shared memory in a fixed order), and one producer warp
-// whose elected lane draws the items, polls their dependencies and stages the input tiles of the next
-// step with bulk asynchronous copies (cp.async.bulk + mbarrier) while the groups compute.
+// Block = two compute groups of 256 threads that take half of the coils of an item each (the coil sum
+// of P3 is completed through shared memory in a fixed order) and a producer warpgroup with one elected
+// lane per group: the first draws the items; each polls the item's dependency and stages the input
+// tiles of its group one step ahead with tiled TMA copies (cp.async.bulk.tensor + mbarrier) while the
+// group computes.  A group owns three 32 KB buffers A | B | C.  The transposition between the row-wise
+// and the column-wise transform happens in place in the staged tile itself (a thread rewrites the column
+// it read; a warp rewrites its own two rows with an XOR-swizzled 16 x 16 exchange), so a step needs one
+// group-wide barrier, and the tile of step s + 1 arrives in the other buffer meanwhile:
+//   P1  x tile -> C once; S tiles alternate A, B      P2  BY rows -> A | B (+ mask rows once)
+//   P3  W tiles alternate B, C; S tile -> A; the x rows for the update follow in the W alternation
 #pragma once
 #include "size_ops.cuh"
 #include <cuda.h>          // CUtensorMap (type only; the encoder is looked up at run time)
@@ -45,11 +51,11 @@ struct FusedArgs {
 
 namespace fused {
 
-constexpr int NZ = 256, RY = 16, GT = 256, ES = 272;     // ES: padded row of the exchange tile (16 * 17)
+constexpr int NZ = 256, RY = 16, GT = 256;
 constexpr int CONSUMERS = 2 * GT, THREADS = CONSUMERS + 128;   // four compute warpgroups + the producer's
 constexpr int REGS_PRODUCER = 24, REGS_COMPUTE = 112;           // register split after the kernel has started
 constexpr int TILE = RY * NZ;                             // complex values of a staged tile (32 KB)
-constexpr int GROUP_ELEMS = 2 * TILE + RY * ES;           // bufA | bufB | E
+constexpr int GROUP_ELEMS = 3 * TILE;                     // A | B | C
 constexpr size_t SMEM_BYTES = sizeof(cf) * 2 * GROUP_ELEMS + 256;
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -92,6 +98,11 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, in
     asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
                  ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d_hint(void* dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3,
+                                                 unsigned long long* bar, unsigned long long policy) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void named_bar(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void st_keep(cf* p, cf v, unsigned long long pol) {      // workspace store, kept in L2
     asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1,%2}, %3;" ::"l"(p), "f"(v.x), "f"(v.y), "l"(pol) : "memory");
@@ -110,7 +121,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned pari
 }
 
 struct Shared {                      // control block behind the tiles
-    unsigned long long full[2][2], empty[2][2];       // [group][A / B]
+    unsigned long long full[2][3], empty[2][3];       // [group][A / B / C]
     unsigned long long item_full[2], item_empty[2];
     int item[2];                                      // item number of the slot (bit 30: withheld)
     int dead[2];                                      // group gave up (sticky)
@@ -132,7 +143,7 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
     using namespace fused;
     constexpr int N1 = RY * BY;
     static_assert(BY >= 2 && BY <= 24 && BY % 2 == 0, "radix of the middle pass (even: the half shift of ky keeps ky mod RY)");
-    static_assert(BY * NZ * 8 + BY * NZ * 4 <= 2 * TILE * 8, "tile and mask rows of the middle pass fit the two buffers");
+    static_assert(BY * NZ * 8 + BY * NZ * 4 <= 2 * TILE * 8, "tile and mask rows of the middle pass fit buffers A | B");
     extern __shared__ __align__(128) float2 fsmem[];
     float2* const smem = fsmem;
     Shared* sh = reinterpret_cast<Shared*>(smem + 2 * GROUP_ELEMS);
@@ -140,8 +151,8 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
 
     if (tid == 0) {
         for (int g = 0; g < 2; ++g)
-            for (int b = 0; b < 2; ++b) { mbar_init(&sh->full[g][b], 1); mbar_init(&sh->empty[g][b], GT / 32); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sh->item_full[s], 1); mbar_init(&sh->item_empty[s], 2); sh->stop_flag[s] = 0; }
+            for (int b = 0; b < 3; ++b) { mbar_init(&sh->full[g][b], 1); mbar_init(&sh->empty[g][b], GT / 32); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sh->item_full[s], 1); mbar_init(&sh->item_empty[s], 3); sh->stop_flag[s] = 0; }
         sh->dead[0] = sh->dead[1] = 0; sh->prod_dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -152,43 +163,41 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
     const int n_g[2] = {(a.C + 1) / 2, a.C / 2};              // coils of group 0 / 1
     const long long slab_elems = (long long)N1 * NZ;
     int* c1 = a.ctrl + 64; int* c2 = c1 + a.nslabs; int* c3 = c2 + a.nslabs;
+    unsigned long long* stats = reinterpret_cast<unsigned long long*>(a.ctrl + 8);
 
-    auto sens_slab = [&](int gs, int c) -> int {               // last coordinate of tm_sens: S_c of slab gs
-        const int bt = gs / a.n0, i0 = gs - bt * a.n0;
-        const int b = bt / a.T, t = bt - b * a.T;
-        return ((b * a.C + c) * a.Ts + (a.Ts > 1 ? t : 0)) * a.n0 + i0;
-    };
-
-    // The launch gives every thread floor(65536 / 640 / 8) * 8 = 96 registers; the producer's warpgroup
+    // The launch gives every thread floor(65536 / 640 / 8) * 8 = 96 registers; the producers' warpgroup
     // hands most of its share back and the compute warpgroups take 112 each:
     // 128 * 24 + 512 * 112 = 60416 <= 640 * 96 = 61440.
     static_assert(128 * REGS_PRODUCER + CONSUMERS * REGS_COMPUTE <= THREADS * 96, "register split exceeds the launch's registers");
     if (warp >= CONSUMERS / 32) {
-        // =================================== producer ===================================
+        // =================================== producers ===================================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_PRODUCER));
-        if (tid != CONSUMERS) return;
-        unsigned nfill[2][2] = {{0, 0}, {0, 0}};
-        bool dead = false;
-        cf* bufs[2][2];
-        for (int g = 0; g < 2; ++g) { bufs[g][0] = smem + g * GROUP_ELEMS; bufs[g][1] = bufs[g][0] + TILE; }
-        // arms the barrier of the next fill of buffer (g, b) once the consumers have released the fill before
-        auto begin_fill = [&](int g, int b, unsigned bytes) -> bool {
-            const unsigned n = nfill[g][b];
-            if (n > 0 && !mbar_wait(&sh->empty[g][b], (n - 1) & 1, &sh->dead[g], a.limit_ns)) return false;
+        const int g = warp - CONSUMERS / 32;                   // the producer of group g is lane 0 of producer warp g
+        if (g > 1 || lane != 0) return;
+        unsigned nfill[3] = {0, 0, 0};
+        cf* const gbase = smem + g * GROUP_ELEMS;
+        unsigned long long pol_first, pol_last;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
+        const int n = n_g[g], c_first = g * n_g[0];
+
+        // arms the barrier of the next fill of buffer b once the group has released the fill before
+        auto begin_fill = [&](int b, unsigned bytes) -> bool {
+            const unsigned f = nfill[b];
+            if (f > 0 && !mbar_wait(&sh->empty[g][b], (f - 1) & 1, &sh->dead[g], a.limit_ns, &sh->prod_dead)) return false;
             mbar_expect_tx(&sh->full[g][b], bytes);
-            nfill[g][b] = n + 1;
+            nfill[b] = f + 1;
             return true;
         };
         // time spent waiting and number of waits that had to spin, per kind (ctrl + 8: pairs of 64-bit words):
         // 0 ring slot free (P1), 1 first pass of the slab complete (P2), 2 middle pass complete (P3)
-        unsigned long long* stats = reinterpret_cast<unsigned long long*>(a.ctrl + 8);
         auto wait_counter = [&](const int* ctr, int target, int kind) -> bool {
             if (ld_acquire(ctr) >= target) return true;
             const unsigned long long t0 = gtimer();
             bool ok = false;
             for (;;) {
                 if (ld_acquire(ctr) >= target) { ok = true; break; }
-                if (ld_relaxed(a.ctrl + 1) != 0) break;
+                if (ld_relaxed(a.ctrl + 1) != 0 || *(volatile int*)&sh->prod_dead != 0) break;
                 if (gtimer() - t0 > a.limit_ns) break;
                 __nanosleep(64);
             }
@@ -196,104 +205,95 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
             atomicAdd(stats + 2 * kind + 1, 1ull);
             return ok;
         };
+        auto sens_slab = [&](int gs, int c) -> int {           // last coordinate of tm_sens: S_c of slab gs
+            const int bt = gs / a.n0, i0 = gs - bt * a.n0;
+            const int b = bt / a.T, t = bt - b * a.T;
+            return ((b * a.C + c) * a.Ts + (a.Ts > 1 ? t : 0)) * a.n0 + i0;
+        };
 
-        for (unsigned k = 0;; ++k) {
+        bool ok = true;
+        for (unsigned k = 0; ok; ++k) {
             const int slot = k & 1;
-            long long id = atomicAdd(a.ctrl, 1);
-            if (id > total) id = total;
-            int word = (int)id;
-            if (id < total && a.withhold >= 0 && id == a.withhold) word |= 1 << 30;
-            // publish the item to the groups
-            if (k >= 2 && !mbar_wait(&sh->item_empty[slot], ((k >> 1) - 1) & 1, &sh->dead[0], a.limit_ns, &sh->dead[1])) dead = true;
-            if (dead) { sh->prod_dead = 1; break; }              // the groups learn it from the flag
-            sh->item[slot] = word;
-            mbar_arrive(&sh->item_full[slot]);
+            int word;
+            if (g == 0) {
+                // draw the next item and publish it to both groups and to the other producer
+                long long id = atomicAdd(a.ctrl, 1);
+                if (id > total) id = total;
+                word = (int)id;
+                if (id < total && a.withhold >= 0 && id == a.withhold) word |= 1 << 30;
+                if (k >= 2 && !mbar_wait(&sh->item_empty[slot], ((k >> 1) - 1) & 1, &sh->dead[0], a.limit_ns, &sh->dead[1])) { ok = false; break; }
+                sh->item[slot] = word;
+                mbar_arrive(&sh->item_full[slot]);
+            } else {
+                if (!mbar_wait(&sh->item_full[slot], (k >> 1) & 1, &sh->prod_dead, a.limit_ns, &sh->dead[1])) { ok = false; break; }
+                word = *(volatile int*)&sh->item[slot];
+                mbar_arrive(&sh->item_empty[slot]);
+            }
+            const long long id = word & ~(1 << 30);
             if (id >= total) break;
             if (word >> 30) continue;
-
             const int period = (int)(id / per_period), q = (int)(id % per_period);
-            bool ok = true;
             if (q < BY) {
-                // ---- P3(gs, j): per step W tile -> B, S tile -> A; at the end the x rows of each group's half -> B
+                // ---- P3(gs, j): per step W tile -> B / C alternating, S tile -> A; then the x tile in the W alternation
                 const int gs = period - a.L3, j = q;
                 if (gs < 0 || gs >= a.nslabs) continue;
                 ok = wait_counter(c2 + gs, RY, 2);
                 asm volatile("fence.proxy.async;" ::: "memory");
                 const int rs = gs % a.R;
-                for (int s = 0; ok && s < n_g[0]; ++s) {
-                    for (int g = 0; ok && g < 2; ++g) {
-                        if (s >= n_g[g]) continue;
-                        const int c = g * n_g[0] + s;
-                        if (!(ok = begin_fill(g, 1, TILE * 8))) break;
-                        tma_load_4d(bufs[g][1], &tm_ring, 0, j, 0, rs * a.C + c, &sh->full[g][1]);
-                    }
-                    for (int g = 0; ok && g < 2; ++g) {
-                        if (s >= n_g[g]) continue;
-                        const int c = g * n_g[0] + s;
-                        if (!(ok = begin_fill(g, 0, TILE * 8))) break;
-                        tma_load_4d(bufs[g][0], &tm_sens, 0, j, 0, sens_slab(gs, c), &sh->full[g][0]);
-                    }
+                for (int s = 0; ok && s < n; ++s) {
+                    const int wb = 1 + (s & 1);
+                    if (!(ok = begin_fill(wb, TILE * 8))) break;
+                    tma_load_4d_hint(gbase + wb * TILE, &tm_ring, 0, j, 0, rs * a.C + c_first + s, &sh->full[g][wb], pol_first);
+                    if (!(ok = begin_fill(0, TILE * 8))) break;
+                    tma_load_4d_hint(gbase, &tm_sens, 0, j, 0, sens_slab(gs, c_first + s), &sh->full[g][0], pol_first);
                 }
-                for (int g = 0; ok && g < 2; ++g) {            // the x rows for the update (each group uses its half)
-                    if (!(ok = begin_fill(g, 1, TILE * 8))) break;
-                    tma_load_4d(bufs[g][1], &tm_x, 0, j, 0, gs, &sh->full[g][1]);
+                if (ok) {
+                    const int xb = 1 + (n & 1);
+                    if ((ok = begin_fill(xb, TILE * 8))) tma_load_4d_hint(gbase + xb * TILE, &tm_x, 0, j, 0, gs, &sh->full[g][xb], pol_first);
                 }
             } else if (q < BY + RY) {
-                // ---- P2(gs, k0): per step the BY rows of (c, k0) -> A | B; with the first step the mask rows
+                // ---- P2(gs, k0): per step the BY rows of (c, k0) -> A | B; with the first step the mask rows behind them
                 const int gs = period - a.L2, k0 = q - BY;
                 if (gs < 0 || gs >= a.nslabs) continue;
                 ok = wait_counter(c1 + gs, BY, 1);
                 asm volatile("fence.proxy.async;" ::: "memory");
                 const int rs = gs % a.R;
                 const int bt = gs / a.n0;
-                for (int s = 0; ok && s < n_g[0]; ++s) {
-                    for (int g = 0; ok && g < 2; ++g) {
-                        if (s >= n_g[g]) continue;
-                        const int c = g * n_g[0] + s;
-                        const cf* src = a.W + (((long long)rs * a.C + c) * RY + k0) * BY * NZ;
-                        constexpr int ROWS_A = BY < RY ? BY : RY, ROWS_B = BY - ROWS_A;
-                        const unsigned bytes_b = ROWS_B * NZ * 8 + (s == 0 ? BY * NZ * 4 : 0);
-                        if (bytes_b > 0) {
-                            if (!(ok = begin_fill(g, 1, bytes_b))) break;
-                            if (ROWS_B > 0) bulk_load(bufs[g][1], src + ROWS_A * NZ, ROWS_B * NZ * 8, &sh->full[g][1]);
-                            if (s == 0) tma_load_4d(bufs[g][0] + BY * NZ, &tm_mask, 0, k0, 0, bt, &sh->full[g][1]);
-                        }
-                        if (!(ok = begin_fill(g, 0, ROWS_A * NZ * 8))) break;
-                        bulk_load(bufs[g][0], src, ROWS_A * NZ * 8, &sh->full[g][0]);
+                constexpr int ROWS_A = BY < RY ? BY : RY, ROWS_B = BY - ROWS_A;
+                for (int s = 0; ok && s < n; ++s) {
+                    const cf* src = a.W + (((long long)rs * a.C + c_first + s) * RY + k0) * BY * NZ;
+                    const unsigned bytes_b = ROWS_B * NZ * 8 + (s == 0 ? BY * NZ * 4 : 0);
+                    if (bytes_b > 0) {
+                        if (!(ok = begin_fill(1, bytes_b))) break;
+                        if (ROWS_B > 0) bulk_load(gbase + TILE, src + ROWS_A * NZ, ROWS_B * NZ * 8, &sh->full[g][1]);
+                        if (s == 0) tma_load_4d(gbase + BY * NZ, &tm_mask, 0, k0, 0, bt, &sh->full[g][1]);
                     }
+                    if (!(ok = begin_fill(0, ROWS_A * NZ * 8))) break;
+                    bulk_load(gbase, src, ROWS_A * NZ * 8, &sh->full[g][0]);
                 }
             } else {
-                // ---- P1(gs, j): x tile -> B, then per step S tile -> A
+                // ---- P1(gs, j): x tile -> C, then per step S tile -> A / B alternating
                 const int gs = period, j = q - BY - RY;
-                if (gs >= a.nslabs) continue;
+                if (gs >= a.nslabs || n == 0) continue;
                 if (gs >= a.R) ok = wait_counter(c3 + gs - a.R, BY, 0);
-                for (int g = 0; ok && g < 2; ++g) {
-                    if (n_g[g] == 0) continue;
-                    if (!(ok = begin_fill(g, 1, TILE * 8))) break;
-                    tma_load_4d(bufs[g][1], &tm_x, 0, j, 0, gs, &sh->full[g][1]);
+                if (ok && (ok = begin_fill(2, TILE * 8))) tma_load_4d(gbase + 2 * TILE, &tm_x, 0, j, 0, gs, &sh->full[g][2]);
+                for (int s = 0; ok && s < n; ++s) {
+                    const int sb = s & 1;
+                    if (!(ok = begin_fill(sb, TILE * 8))) break;
+                    tma_load_4d(gbase + sb * TILE, &tm_sens, 0, j, 0, sens_slab(gs, c_first + s), &sh->full[g][sb]);
                 }
-                for (int s = 0; ok && s < n_g[0]; ++s)
-                    for (int g = 0; ok && g < 2; ++g) {
-                        if (s >= n_g[g]) continue;
-                        const int c = g * n_g[0] + s;
-                        if (!(ok = begin_fill(g, 0, TILE * 8))) break;
-                        tma_load_4d(bufs[g][0], &tm_sens, 0, j, 0, sens_slab(gs, c), &sh->full[g][0]);
-                    }
-            }
-            if (!ok) {
-                // gave up: raise the error word, tell the groups, start nothing more
-                atomicExch(a.ctrl + 1, 1);
-                sh->prod_dead = 1;
-                break;
             }
         }
+        if (!ok) {                                   // gave up: raise the error word, tell everyone in the block
+            atomicExch(a.ctrl + 1, 1);
+            sh->prod_dead = 1;
+        }
         // copies that were started must have landed before the block may end
-        for (int g = 0; g < 2; ++g)
-            for (int b = 0; b < 2; ++b)
-                if (nfill[g][b] > 0) {
-                    volatile int never = 0;
-                    mbar_wait(&sh->full[g][b], (nfill[g][b] - 1) & 1, &never, a.limit_ns);
-                }
+        for (int b = 0; b < 3; ++b)
+            if (nfill[b] > 0) {
+                volatile int never = 0;
+                mbar_wait(&sh->full[g][b], (nfill[b] - 1) & 1, &never, a.limit_ns);
+            }
         return;
     }
 
@@ -301,31 +301,33 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_COMPUTE));
     const int g = warp >> 3;                       // group
     const int gt = tid & (GT - 1);                 // thread of the group
-    const int r = gt >> 4, a16 = gt & 15;          // row-owned layout: row and position inside the 16 x 16 split of kz
-    cf* bufA = smem + g * GROUP_ELEMS;
-    cf* bufB = bufA + TILE;
-    cf* E = bufB + TILE;
-    cf* Eother = smem + (g ^ 1) * GROUP_ELEMS + 2 * TILE;
+    const int r = gt >> 4, a16 = gt & 15;          // row-owned layout: row, and position in the 16 x 16 split of kz
+    cf* const gbase = smem + g * GROUP_ELEMS;      // A | B | C
+    cf* const obase = smem + (g ^ 1) * GROUP_ELEMS;
     const int gbar = 1 + g;
-    unsigned nuse[2] = {0, 0};                     // fills of A / B consumed so far
+    unsigned nuse[3] = {0, 0, 0};                  // fills of A / B / C consumed so far
     bool dead = false;                             // the whole group shares this value at every barrier
     unsigned long long keep_policy;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep_policy));
 
-    // the elected thread waits for the next fill of buffer b; the result reaches the group at the barrier that follows
-    unsigned long long* stats = reinterpret_cast<unsigned long long*>(a.ctrl + 8);
+    // every warp waits for the next fill of buffer b through its first lane (bounded); a warp that gave up keeps
+    // running the same control flow without waiting and without storing
     auto wait_full = [&](int b) {
-        if (gt == 0 && !dead) {
-            if (!mbar_try(&sh->full[g][b], nuse[b] & 1)) {       // the tile has not landed yet: count the wait (kinds 3: A, 4: B)
+        int failed = 0;
+        if (lane == 0 && !dead) {
+            if (!mbar_try(&sh->full[g][b], nuse[b] & 1)) {
                 const unsigned long long t0 = gtimer();
-                if (!mbar_wait(&sh->full[g][b], nuse[b] & 1, &sh->prod_dead, a.limit_ns)) sh->dead[g] = 1;
-                atomicAdd(stats + 2 * (3 + b), gtimer() - t0);
-                atomicAdd(stats + 2 * (3 + b) + 1, 1ull);
+                if (!mbar_wait(&sh->full[g][b], nuse[b] & 1, &sh->prod_dead, a.limit_ns, &sh->dead[g])) { sh->dead[g] = 1; failed = 1; }
+                if (gt == 0) {                                   // not landed when needed: count the wait (kinds 3: A, 4: B or C)
+                    atomicAdd(stats + 2 * (b == 0 ? 3 : 4), gtimer() - t0);
+                    atomicAdd(stats + 2 * (b == 0 ? 3 : 4) + 1, 1ull);
+                }
             }
         }
+        dead = dead || (__shfl_sync(0xffffffffu, failed, 0) != 0);
         ++nuse[b];
     };
-    auto release = [&](int b) {                    // this warp has read the buffer
+    auto release = [&](int b) {                    // this warp has finished with the buffer
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh->empty[g][b]);
     };
@@ -333,6 +335,8 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
         named_bar(gbar, GT);
         dead = dead || (*(volatile int*)&sh->dead[g] != 0);
     };
+    // 16 x 16 exchange inside one row of 256 values, conflict-free without padding: element (p, q) lives at 16 p + (q ^ p)
+    auto xs = [&](int p, int q) -> int { return 16 * p + (q ^ p); };
 
     for (unsigned k = 0;; ++k) {
         const int slot = k & 1;
@@ -354,95 +358,109 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
         }
         const int period = (int)(id / per_period), q = (int)(id % per_period);
         int* done_ctr = nullptr;
+        bool release_a_after_close = false;
+        const int n = n_g[g], c_first = g * n_g[0];
 
         if (q < BY) {
             // ------------------------------ P3(gs, j) ------------------------------
             const int gs = period - a.L3;
             const bool live = !withheld && gs >= 0 && gs < a.nslabs;
-            cf acc[RY];
-#pragma unroll
-            for (int m = 0; m < RY; ++m) acc[m] = make_float2(0.f, 0.f);
             if (live) {
+                cf acc[RY];
+#pragma unroll
+                for (int m = 0; m < RY; ++m) acc[m] = make_float2(0.f, 0.f);
                 cf twz[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) twz[e] = unit_root_fwd<NZ>((a16 * e) % NZ);
-                for (int s = 0; s < n_g[g]; ++s) {
-                    wait_full(1);
-                    group_sync();
+                cf* const S = gbase;
+                for (int s = 0; s < n; ++s) {
+                    const int wb = 1 + (s & 1);
+                    cf* const row = gbase + wb * TILE + r * NZ;          // this thread's row of the W tile
+                    wait_full(wb);         // the column reads of the step before used the other W buffer
+                    // ---- kz inverse of the warp's two rows, in place ----
                     cf w[16];
 #pragma unroll
-                    for (int k1 = 0; k1 < 16; ++k1) w[k1] = bufB[r * NZ + a16 + 16 * k1];
-                    release(1);
+                    for (int k1 = 0; k1 < 16; ++k1) w[k1] = row[a16 + 16 * k1];
                     Dft<16, +1>::run(w);                               // k1 -> a'
 #pragma unroll
                     for (int e = 1; e < 16; ++e) w[e] = cmulc(w[e], twz[e]);
+                    __syncwarp();
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) E[r * ES + a16 * 17 + e] = w[e];
+                    for (int e = 0; e < 16; ++e) row[xs(a16, e)] = w[e];
                     __syncwarp();
                     cf u[16];
 #pragma unroll
-                    for (int k2 = 0; k2 < 16; ++k2) u[k2] = E[r * ES + k2 * 17 + a16];
+                    for (int k2 = 0; k2 < 16; ++k2) u[k2] = row[xs(k2, a16)];
                     Dft<16, +1>::run(u);                               // k2 -> b
                     __syncwarp();
 #pragma unroll
-                    for (int b = 0; b < 16; ++b) E[r * ES + a16 + 16 * b] = u[b];
+                    for (int b = 0; b < 16; ++b) row[a16 + 16 * b] = u[b];
                     wait_full(0);
-                    group_sync();
+                    named_bar(gbar, GT);
+                    // ---- inverse radix-RY across the rows, conj(S) and the coil sum: one kz position per thread ----
                     cf v[RY];
+                    const cf* const col = gbase + wb * TILE + gt;
 #pragma unroll
-                    for (int k0 = 0; k0 < RY; ++k0) v[k0] = E[k0 * ES + gt];
+                    for (int k0 = 0; k0 < RY; ++k0) v[k0] = col[k0 * NZ];
+                    release(wb);
                     Dft<RY, +1>::run(v);                               // k0 -> m
 #pragma unroll
                     for (int m = 0; m < RY; ++m) {
-                        const cf sv = bufA[m * NZ + gt];
+                        const cf sv = S[m * NZ + gt];
                         acc[m].x = fmaf(sv.x, v[m].x, fmaf(sv.y, v[m].y, acc[m].x));
                         acc[m].y = fmaf(sv.x, v[m].y, fmaf(-sv.y, v[m].x, acc[m].y));
                     }
-                    release(0);
+                    if (s + 1 < n) release(0);          // after the last step buffer A carries the partial sums below
                 }
-                // partial coil sums of this group; a thread only ever touches its own column of E here
+                // partial coil sums of this group into buffer A (a thread only touches its own column), x tile in the W alternation
+                if (n > 0) {
 #pragma unroll
-                for (int m = 0; m < RY; ++m) E[m * ES + gt] = acc[m];
-                wait_full(1);
+                    for (int m = 0; m < RY; ++m) S[m * NZ + gt] = acc[m];
+                } else {
+#pragma unroll
+                    for (int m = 0; m < RY; ++m) S[m * NZ + gt] = make_float2(0.f, 0.f);
+                }
+                wait_full(1 + (n & 1));
             }
             if (dead && gt == 0) sh->stop_flag[slot] = 1;
             named_bar(3, CONSUMERS);
             dead = dead || (*(volatile int*)&sh->dead[g] != 0);
             if (live) {
                 // group g completes rows m in [g RY/2, (g+1) RY/2): group 0's partial sum + group 1's, then the update
-                const cf* E0 = g == 0 ? E : Eother;
-                const cf* E1 = g == 0 ? Eother : E;
+                const cf* P0 = g == 0 ? gbase : obase;
+                const cf* P1 = g == 0 ? obase : gbase;
+                const cf* X = gbase + (1 + (n & 1)) * TILE;
                 const long long xo = (long long)gs * slab_elems + (long long)q * NZ + gt;
 #pragma unroll
                 for (int mm = 0; mm < RY / 2; ++mm) {
                     const int m = g * (RY / 2) + mm;
-                    const cf p0 = E0[m * ES + gt], p1 = E1[m * ES + gt];
-                    const cf xv = bufB[m * NZ + gt];
+                    const cf p0 = P0[m * NZ + gt], p1 = P1[m * NZ + gt];
+                    const cf xv = X[m * NZ + gt];
                     const float sx = p0.x + p1.x, sy = p0.y + p1.y;
                     if (!dead) a.out[xo + (long long)BY * m * NZ] = make_float2(fmaf(-a.eta, sx, xv.x), fmaf(-a.eta, sy, xv.y));
                 }
-                release(1);
+                release(1 + (n & 1));
                 done_ctr = c3 + gs;
+                release_a_after_close = n > 0;      // the other group reads this group's partial sums until the closing barrier
             }
         } else if (q < BY + RY) {
             // ------------------------------ P2(gs, k0) ------------------------------
             const int gs = period - a.L2, k0 = q - BY;
             const bool live = !withheld && gs >= 0 && gs < a.nslabs;
-            if (live) {
+            if (live && n > 0) {
                 const int rs = gs % a.R;
                 cf twy[BY];
 #pragma unroll
                 for (int j = 0; j < BY; ++j) twy[j] = unit_root_fwd<N1>((j * k0) % N1);
                 float wts[BY];
-                const float* mrows = reinterpret_cast<const float*>(bufA + BY * NZ);
-                for (int s = 0; s < n_g[g]; ++s) {
-                    const int c = g * n_g[0] + s;
+                const float* mrows = reinterpret_cast<const float*>(gbase + BY * NZ);
+                for (int s = 0; s < n; ++s) {
+                    const int c = c_first + s;
                     wait_full(0);
                     if (BY > RY || s == 0) wait_full(1);
-                    group_sync();
                     cf cv[BY];
 #pragma unroll
-                    for (int j = 0; j < BY; ++j) cv[j] = bufA[j * NZ + gt];        // rows beyond RY continue into bufB
+                    for (int j = 0; j < BY; ++j) cv[j] = gbase[j * NZ + gt];        // rows beyond RY continue into buffer B
                     if (s == 0) {
 #pragma unroll
                         for (int k1 = 0; k1 < BY; ++k1) {         // the staged rows are ky = k0 + RY k1' in natural order; the raw index needs the half shift
@@ -466,51 +484,52 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
                         for (int j = 0; j < BY; ++j) st_keep(dst + j * NZ, cv[j], keep_policy);
                     }
                 }
-                done_ctr = c2 + gs;
             }
+            if (live) done_ctr = c2 + gs;
             if (dead && gt == 0) sh->stop_flag[slot] = 1;
             named_bar(3, CONSUMERS);
-            dead = dead || (*(volatile int*)&sh->dead[g] != 0);
         } else {
             // ------------------------------ P1(gs, j) ------------------------------
             const int gs = period, j = q - BY - RY;
             const bool live = !withheld && gs < a.nslabs;
-            if (live && n_g[g] > 0) {
+            if (live && n > 0) {
                 const int rs = gs % a.R;
                 cf twz[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) twz[e] = unit_root_fwd<NZ>((a16 * e) % NZ);
-                wait_full(1);
-                group_sync();
+                wait_full(2);
                 cf xr[RY];
 #pragma unroll
-                for (int m = 0; m < RY; ++m) xr[m] = bufB[m * NZ + gt];
-                release(1);
-                for (int s = 0; s < n_g[g]; ++s) {
-                    const int c = g * n_g[0] + s;
-                    wait_full(0);
-                    group_sync();                                       // also: the row reads of the step before are complete
+                for (int m = 0; m < RY; ++m) xr[m] = gbase[2 * TILE + m * NZ + gt];
+                release(2);
+                for (int s = 0; s < n; ++s) {
+                    const int c = c_first + s, sb = s & 1;
+                    cf* const tile = gbase + sb * TILE;
+                    wait_full(sb);
+                    // ---- S x and the radix-RY transform across the rows: one kz position per thread, in place ----
                     cf v[RY];
 #pragma unroll
-                    for (int m = 0; m < RY; ++m) v[m] = cmul(bufA[m * NZ + gt], xr[m]);
-                    release(0);
+                    for (int m = 0; m < RY; ++m) v[m] = cmul(tile[m * NZ + gt], xr[m]);
                     Dft<RY, -1>::run(v);                               // m -> k0
 #pragma unroll
-                    for (int k0 = 0; k0 < RY; ++k0) E[k0 * ES + gt] = v[k0];
-                    group_sync();
+                    for (int k0 = 0; k0 < RY; ++k0) tile[k0 * NZ + gt] = v[k0];
+                    named_bar(gbar, GT);
+                    // ---- kz transform of the warp's two rows, in place, then out to the ring ----
+                    cf* const row = tile + r * NZ;
                     cf u[16];
 #pragma unroll
-                    for (int b = 0; b < 16; ++b) u[b] = E[r * ES + a16 + 16 * b];
+                    for (int b = 0; b < 16; ++b) u[b] = row[a16 + 16 * b];
                     Dft<16, -1>::run(u);                               // b -> k2
 #pragma unroll
                     for (int e = 1; e < 16; ++e) u[e] = cmul(u[e], twz[e]);
                     __syncwarp();
 #pragma unroll
-                    for (int k2 = 0; k2 < 16; ++k2) E[r * ES + k2 * 17 + a16] = u[k2];
+                    for (int k2 = 0; k2 < 16; ++k2) row[xs(k2, a16)] = u[k2];
                     __syncwarp();
                     cf w[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) w[e] = E[r * ES + a16 * 17 + e];
+                    for (int e = 0; e < 16; ++e) w[e] = row[xs(a16, e)];
+                    release(sb);
                     Dft<16, -1>::run(w);                               // a' -> k1
                     cf* dst = a.W + ((((long long)rs * a.C + c) * RY + r) * BY + j) * NZ + a16;
                     if (!dead) {
@@ -522,10 +541,12 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
             if (live) done_ctr = c1 + gs;
             if (dead && gt == 0) sh->stop_flag[slot] = 1;
             named_bar(3, CONSUMERS);
-            dead = dead || (*(volatile int*)&sh->dead[g] != 0);
         }
         // closing barrier of the item: every store of the item precedes the count that publishes it
+        dead = dead || (*(volatile int*)&sh->dead[g] != 0);
+        if (dead && lane == 0) sh->stop_flag[slot] = 1;
         named_bar(3, CONSUMERS);
+        if (release_a_after_close) release(0);
         const bool stop_now = *(volatile int*)&sh->stop_flag[slot] != 0;
         if (tid == 0 && done_ctr != nullptr && !stop_now) { __threadfence(); red_release(done_ctr, 1); }
         if (stop_now) {

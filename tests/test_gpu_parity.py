@@ -224,6 +224,19 @@ def test_workload_knee3d_full_size(oracle):
     assert_close(gotv, refv, inp["g"], "knee3d vjp")
 
 
+def test_workload_knee3d_full_size_general_mask(oracle):
+    """The same volume with its mask handed over as a general (B, T, n0, n1, n2) array: the arbitrary-mask
+    path (three transformed axes on a coil-volume workspace) at full size."""
+    w, d, inp, mask, y = workload_case(oracle, "knee3d", MASK_FULL)
+    got = run_gpu(inp["x"], y, inp["sens"], mask, w.eta, 3, 0, MASK_FULL)
+    ref = oracle.dc_forward(inp["x"], y, inp["sens"], mask, w.eta, d, nthreads=8)
+    assert_close(got, ref, inp["x"], "knee3d forward, general mask")
+    del ref, got
+    gotv = run_gpu(inp["g"], None, inp["sens"], mask, w.eta, 3, 0, MASK_FULL)
+    refv = oracle.dc_vjp(inp["g"], inp["sens"], mask, w.eta, d, nthreads=8)
+    assert_close(gotv, refv, inp["g"], "knee3d vjp, general mask")
+
+
 def test_chained_iterations_match_oracle(oracle):
     """Unrolled chain as the cine workload runs it: x_{i+1} = DC(x_i), then g_i = VJP(g_{i+1})."""
     w = wl.scaled(wl.WORKLOADS["cine"], frames=4, n=(1, 48, 40), chain=4)

@@ -12,6 +12,7 @@ other test.
 import numpy as np
 import pytest
 
+from oracle.oracle import Dims
 from tests.gpu_common import assert_close
 
 pytestmark = pytest.mark.gpu
@@ -27,7 +28,7 @@ def _case(seed, B, C, T, rank, n):
 
 
 @pytest.mark.parametrize("rank,n", [(2, (1, 64, 160)), (3, (8, 20, 32))])
-def test_static_scratch_forward_matches_workspace_forward_twice(rank, n):
+def test_static_scratch_forward_matches_workspace_forward_twice(oracle, rank, n):
     import torch
     import paper_2207_08393_b200 as g
     dev = torch.device("cuda:0")
@@ -47,6 +48,14 @@ def test_static_scratch_forward_matches_workspace_forward_twice(rank, n):
                                                                         stream=torch.cuda.current_stream()))
         torch.cuda.synchronize()
         assert_close(out.cpu().numpy(), ref.cpu().numpy().astype(np.complex128), x, "static scratch, call %d" % call)
+        # element by element against the CPU oracle as well, and no device memory taken by a repeated call
+        assert_close(out.cpu().numpy(), oracle.dc_forward(x, y, sens, mask, eta, Dims(B, C, T, rank, n, 0, 1), nthreads=8), x,
+                     "static scratch against the oracle, call %d" % call)
+        free_before = torch.cuda.mem_get_info()[0]
+        g.gleam_dc_forward_static(tx, ty, ts, tm, eta, out, g.make_dims(B, C, T, rank, n,
+                                                                        stream=torch.cuda.current_stream()))
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
 
 
 def test_static_scratch_rejects_problems_beyond_its_size():

@@ -480,6 +480,7 @@ def run_ours(args, w):
     # ---- roofline --------------------------------------------------------------------------------
     sm_mhz = peaks["sm_max_mhz"]
     alu_peak = fp32_peak_tflops(sm_mhz)
+    alu_measured = g.gleam_measure_fp32_peak(out, stream)      # independent FMA chains, best of four launches
     dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     kd = kernels[dom]
     t_hbm = kd["gbs"] / peaks["hbm_gbs"]
@@ -496,7 +497,8 @@ def run_ours(args, w):
         nbytes, flops = call_roofline(w, with_y)
         t_b, t_f = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (alu_peak * 1e12)
         ns[name] = {"min_bytes": nbytes, "fft_flops": flops, "hbm_us": t_b * 1e6, "fp32_us": t_f * 1e6,
-                    "measured_us": ms * 1e3, "frac": max(t_b, t_f) / (ms * 1e-3)}
+                    "measured_us": ms * 1e3, "frac": max(t_b, t_f) / (ms * 1e-3),
+                    "frac_with_measured_fp32_peak": max(t_b, flops / (alu_measured * 1e12)) / (ms * 1e-3)}
 
     # ---- CPU baseline: the oracle, once, on the host cores of the machine ---------------------------
     cpu = None
@@ -535,6 +537,8 @@ def run_ours(args, w):
         "gpu_launches": int(launches),
         "roofline": roof,
         "call_roofline": ns,
+        "fp32_peak": {"derived_tflops": alu_peak, "measured_tflops": alu_measured,
+                      "how": "derived: 148 SMs x 128 lanes x 2 flop x sm_max_mhz; measured: independent FMA chains, no memory traffic"},
         "prepared_chain": prepared,
         "warm_l2": warm,
         "two_channel_layout": layout_cost,

@@ -124,6 +124,13 @@ GLEAM_API int gleam_dc_workspace_size(const gleam_dims* dims, uint64_t* bytes);
 GLEAM_API int gleam_dc_check_status(const gleam_dims* dims);
 
 /*
+ * Which kernels the separable 3-D path uses for phase-encode extents (n1, n2): the number of rows RY a block
+ * of the row-tile kernels holds (n1 = RY * BY; every pass over the workspace contiguous), or 0 when the pair
+ * has no row-tile kernels and the general strided middle pass is used.  Informational.
+ */
+GLEAM_API int32_t gleam_dc_rowtile_split(int32_t n1, int32_t n2);
+
+/*
  * Selects (on != 0) or deselects the persistent kernel for the problem class described above; the default
  * is off unless the environment holds GLEAM_FUSED=1, because the three whole-volume passes measure faster
  * on one B200.  Process-wide; call it before gleam_dc_workspace_size (the scratch layout depends on it).
@@ -318,6 +325,10 @@ enum {
     GLEAM_K_CLASSES = 11
 };
 GLEAM_API uint64_t gleam_dc_launch_count(void);
+/* FP32 FMA throughput of the current device in TFLOP/s (2 flop per FMA), from a kernel of independent FMA
+ * chains without memory traffic, best of four timed launches: the measured ALU peak the benchmark reports
+ * beside the nominal one.  scratch4: at least 4 device bytes (never written).  Synchronises the stream. */
+GLEAM_API int gleam_measure_fp32_peak(void* scratch4, void* stream, double* tflops);
 GLEAM_API int gleam_dc_profile_begin(void);
 GLEAM_API int gleam_dc_profile_end(float* ms, uint32_t* launches, int32_t n_classes);
 

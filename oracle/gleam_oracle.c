@@ -468,18 +468,6 @@ static int normal_op(const zc* p, const float* sens, const float* mask, const od
     return rc;
 }
 
-/* out = A^H A p  (exported for the pins: the dense matrix of H is assembled from it) */
-int oracle_normal_op(const zc* p, const float* sens, const float* mask, const int64_t* dims, zc* out, int nthreads)
-{
-    odims o;
-    if (parse_dims(dims, &o) != ORACLE_OK || !p || !sens || !mask || !out) return ORACLE_ERR_ARG;
-    zc* kwork = (zc*)malloc(sizeof(zc) * (size_t)(o.B * o.C * o.T * o.V));
-    if (!kwork) return ORACLE_ERR_MEM;
-    const int rc = normal_op(p, sens, mask, &o, kwork, out, nthreads);
-    free(kwork);
-    return rc;
-}
-
 /* n_iter CG steps on (A^H A + mu I) x = b from x = 0.  b is overwritten (it becomes the residual).
  * Every batch example is its own system (A is block diagonal over the batch): the inner products,
  * alpha and beta are taken per example, over its frames and voxels, so a result does not depend

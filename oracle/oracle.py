@@ -52,8 +52,6 @@ def _load():
         lib.oracle_apply_AH.restype = i32
         lib.oracle_dc.argtypes = [p, p, p, p, dbl, p, p, i32]
         lib.oracle_dc.restype = i32
-        lib.oracle_normal_op.argtypes = [p, p, p, p, p, i32]
-        lib.oracle_normal_op.restype = i32
         lib.oracle_modl_cg.argtypes = [p, p, p, p, dbl, i32, p, p, i32]
         lib.oracle_modl_cg.restype = i32
         lib.oracle_modl_cg_vjp.argtypes = [p, p, p, dbl, i32, p, p, i32]
@@ -214,17 +212,6 @@ def dc_vjp(g, sens, mask, eta: float, d: Dims, nthreads: int = 1) -> np.ndarray:
     out = np.empty(d.image_shape(), dtype=np.complex128)
     dd = d.as_array()
     rc = _load().oracle_dc(_ptr(g), None, _ptr(sens), _ptr(mask), float(eta), _ptr(dd), _ptr(out), nthreads)
-    assert rc == 0, rc
-    return out
-
-
-def normal_op(p, sens, mask, d: Dims, nthreads: int = 1) -> np.ndarray:
-    """A^H A p for a double-precision image p."""
-    p = np.ascontiguousarray(np.asarray(p, dtype=np.complex128).reshape(d.image_shape()))
-    sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
-    out = np.empty(d.image_shape(), dtype=np.complex128)
-    dd = d.as_array()
-    rc = _load().oracle_normal_op(_ptr(p), _ptr(sens), _ptr(mask), _ptr(dd), _ptr(out), nthreads)
     assert rc == 0, rc
     return out
 

@@ -54,7 +54,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(BUILD, "kernels_group%d.o" % g)
         jobs.append((["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) +
                      ["-DGLEAM_GROUP=%d" % g, "-c", os.path.join(CSRC, "kernels_group.cu"), "-o", obj], obj))
-    for name in ("gleam_dc", "kernels_pairs", "kernels_fused", "modl_cg"):
+    npair = len(set(re.findall(r"GLEAM_PAIR_GROUP == (\d+)", open(os.path.join(CSRC, "pairs.def")).read())))
+    for g in range(npair):
+        obj = os.path.join(BUILD, "kernels_pairs%d.o" % g)
+        jobs.append((["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) +
+                     ["-DGLEAM_PAIR_GROUP=%d" % g, "-c", os.path.join(CSRC, "kernels_pairs.cu"), "-o", obj], obj))
+    for name in ("gleam_dc", "kernels_fused", "modl_cg"):
         obj = os.path.join(BUILD, name + ".o")
         jobs.append((["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) +
                      ["-c", os.path.join(CSRC, name + ".cu"), "-o", obj], obj))

@@ -38,7 +38,8 @@ EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam
            "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_adjoint",
            "gleam_dc_check_status", "gleam_dc_debug_fused", "gleam_dc_fused_wait_stats", "gleam_dc_set_fused",
            "gleam_dc_grad_eta", "gleam_dc_grad_y", "gleam_dc_grad_workspace_size",
-           "gleam_dc_forward_layout", "gleam_dc_vjp_layout", "gleam_l1_loss", "gleam_l1_loss_workspace_size"]
+           "gleam_dc_forward_layout", "gleam_dc_vjp_layout", "gleam_l1_loss", "gleam_l1_loss_workspace_size",
+           "gleam_measure_fp32_peak", "gleam_dc_rowtile_split"]
 
 KERNEL_CLASSES = ["zmap", "col_z", "row_fused", "row_fwd", "col_mid_sep", "row_inv", "col_mid_full", "col_fwd",
                   "col_inv", "cg_vec", "fused3d"]
@@ -134,6 +135,10 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_l1_loss.restype = i32
         lib.gleam_l1_loss_workspace_size.argtypes = []
         lib.gleam_l1_loss_workspace_size.restype = u64
+        lib.gleam_measure_fp32_peak.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
+        lib.gleam_measure_fp32_peak.restype = i32
+        lib.gleam_dc_rowtile_split.argtypes = [ctypes.c_int32, ctypes.c_int32]
+        lib.gleam_dc_rowtile_split.restype = ctypes.c_int32
         lib.gleam_dc_set_fused.argtypes = [ctypes.c_int32]
         lib.gleam_dc_set_fused.restype = None
         lib.gleam_dc_debug_fused.argtypes = [ctypes.c_int32, u64]
@@ -281,6 +286,20 @@ def gleam_l1_loss_workspace_size() -> int:
 def gleam_l1_loss(x, ref, loss, grad, dims: gleam_dims, layout: int = 0) -> None:
     """loss (device float64 scalar) = mean |x - ref|; grad (optional) = (x - ref)/|x - ref|/N."""
     _check(load_library().gleam_l1_loss(_addr(x), _addr(ref), _addr(loss), _addr(grad), ctypes.byref(dims), int(layout)))
+
+
+def gleam_measure_fp32_peak(scratch, stream=None) -> float:
+    """Measured FP32 FMA peak of the current device in TFLOP/s (independent FMA chains, no memory traffic)."""
+    out = ctypes.c_double(0.0)
+    if stream is not None and not isinstance(stream, int):
+        stream = stream.cuda_stream
+    _check(load_library().gleam_measure_fp32_peak(_addr(scratch), stream or None, ctypes.byref(out)))
+    return float(out.value)
+
+
+def gleam_dc_rowtile_split(n1: int, n2: int) -> int:
+    """Rows per block of the row-tile kernels for phase-encode extents (n1, n2), 0 if the pair has none."""
+    return int(load_library().gleam_dc_rowtile_split(int(n1), int(n2)))
 
 
 def gleam_dc_set_fused(on: bool) -> None:

@@ -136,11 +136,15 @@ warpline_kernel(const RowArgs a) {
                 if (!a.x_planar) {
                     for (int i = lane; i < N / 2; i += 32) cp_async16(sX + ll * N + 2 * i, a.x + xo + 2 * i);
                 } else {
-                    // two-channel layout: the line's real parts, then its imaginary parts, land interleaved
+                    // two-channel layout: the line's real parts and its imaginary parts are two contiguous runs
                     const long long bo = __shfl_sync(0xffffffffu, (long long)b, ll * TPL);
                     const float* xf = reinterpret_cast<const float*>(a.x) + xo + bo * a.plane;
                     float* dst = reinterpret_cast<float*>(sX + ll * N);
-                    for (int i = lane; i < N; i += 32) { dst[2 * i] = xf[i]; dst[2 * i + 1] = xf[a.plane + i]; }
+                    if (N % 4 == 0) {       // staged as two planes of N floats (16-byte copies), read as pairs below
+                        for (int i = lane; i < N / 4; i += 32) { cp_async16(dst + 4 * i, xf + 4 * i); cp_async16(dst + N + 4 * i, xf + a.plane + 4 * i); }
+                    } else {
+                        for (int i = lane; i < N; i += 32) { dst[2 * i] = xf[i]; dst[2 * i + 1] = xf[a.plane + i]; }
+                    }
                 }
             }
             if (MODE == ROW_FUSED) {
@@ -183,11 +187,17 @@ warpline_kernel(const RowArgs a) {
             const cf* cK = sK + buf * KTILE + l * KSTRIDE;
             const cf* gK = use_z ? a.z + k_off + c * k_stride : nullptr;   // this line's compact z row
             const cf* cX = sX + l * N;
+            const bool x_planes = WL::HAS_X && a.x_planar && (N % 4 == 0);       // x staged as two planes of floats
+            auto x_at = [&](int idx) -> cf {
+                if (!x_planes) return cX[idx];
+                const float* xf = reinterpret_cast<const float*>(cX);
+                return make_float2(xf[idx], xf[N + idx]);
+            };
             cf v[R0], u[RL];
             if (MODE != ROW_INV) {
                 if (a0) {
 #pragma unroll
-                    for (int m = 0; m < R0; ++m) v[m] = cmul(cS[j + P::BF0 * m], WL::HAS_X ? cX[j + P::BF0 * m] : xreg[m]);
+                    for (int m = 0; m < R0; ++m) v[m] = cmul(cS[j + P::BF0 * m], WL::HAS_X ? x_at(j + P::BF0 * m) : xreg[m]);
                     Dft<R0, -1>::run(v);
                 }
                 if (P::S == 2) {
@@ -284,7 +294,12 @@ warpline_kernel(const RowArgs a) {
             if (a0 && row_ok) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
-                    const cf xv = WL::HAS_X ? sX[l * N + j + P::BF0 * m] : xreg[m];
+                    cf xv = xreg[m];
+                    if (WL::HAS_X) {
+                        const int idx = j + P::BF0 * m;
+                        const float* xf = reinterpret_cast<const float*>(sX + l * N);
+                        xv = (a.x_planar && (N % 4 == 0)) ? make_float2(xf[idx], xf[N + idx]) : sX[l * N + idx];
+                    }
                     const cf ov = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
                     store_image(a.out, x_off + j + P::BF0 * m, ov, a.out_planar, b, a.plane);
                     if (MODE == ROW_FUSED && a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;

@@ -549,6 +549,22 @@ __global__ void l1_final_kernel(const double* __restrict__ part, int nblocks, do
     }
 }
 
+
+// ---- FP32 peak probe (measurement aid): independent FMA chains, no memory traffic ----
+__global__ void __launch_bounds__(256) fma_peak_kernel(float* sink, int iters, float a, float b) {
+    float v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = (float)(threadIdx.x + i);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = fmaf(v[i], a, b);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s += v[i];
+    if (s == 12345.678f) sink[0] = s;              // never true: keeps the chains alive
+}
+
 struct GradLayout { uint64_t dc_bytes, off_t, off_part, off_W, total; long long ne; int nblocks; };
 static int grad_layout(const gleam_dims* d, GradLayout* G) {
     Layout L;
@@ -655,10 +671,41 @@ GLEAM_API int gleam_dc_fused_wait_stats(const gleam_dims* dims, uint64_t* ns_and
     return GLEAM_OK;
 }
 
+GLEAM_API int32_t gleam_dc_rowtile_split(int32_t n1, int32_t n2) {
+    const gleam::PairOps* p = gleam::find_pair(n1, n2);
+    return p ? p->ry : 0;
+}
+
 GLEAM_API void gleam_dc_set_fused(int32_t on) { gleam::g_fused_on.store(on ? 1 : 0); }
 
 GLEAM_API void gleam_dc_debug_fused(int32_t withhold_item, uint64_t wait_limit_ns) {
     gleam::fused3d_set_debug(withhold_item, wait_limit_ns);
+}
+
+GLEAM_API int gleam_measure_fp32_peak(void* scratch4, void* stream, double* tflops) {
+    if (!scratch4 || !tflops) return GLEAM_ERR_NULL_POINTER;
+    int rc = gleam::check_device_ptr(scratch4);
+    if (rc != GLEAM_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GLEAM_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return GLEAM_ERR_CUDA;
+    const int iters = 1 << 14, blocks = sms * 8;
+    double best = 0.0;
+    for (int rep = 0; rep < 5; ++rep) {
+        cudaEventRecord(e0, s);
+        gleam::fma_peak_kernel<<<blocks, 256, 0, s>>>((float*)scratch4, iters, 0.999f, 0.001f);
+        cudaEventRecord(e1, s);
+        if (cudaEventSynchronize(e1) != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); return GLEAM_ERR_CUDA; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double tf = 2.0 * 16.0 * iters * 256.0 * blocks / (ms * 1e-3) / 1e12;
+        if (rep > 0 && tf > best) best = tf;
+    }
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    *tflops = best;
+    return GLEAM_OK;
 }
 
 GLEAM_API uint64_t gleam_l1_loss_workspace_size(void) { return GRAD_MAX_BLOCKS * sizeof(double); }

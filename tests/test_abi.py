@@ -105,3 +105,31 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         binding.load_library(str(tmp_path / "nope.so"))
+
+
+def test_every_eligible_extent_pair_has_row_tile_kernels(lib):
+    """The separable 3-D path has contiguous row-tile passes for every (n1, n2) whose plans allow them: the
+    library's table against the eligibility rule evaluated here from sizes.def (two-stage split of n1 whose
+    first radix is a multiple of the lines a warp holds of n2; two-stage warp-resident plan of n2; shared memory)."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("gen_pairs", os.path.join(ROOT, "paper_2207_08393_b200", "csrc", "gen_pairs.py"))
+    gp = importlib.util.module_from_spec(spec); spec.loader.exec_module(gp)
+    P = gp.plans()
+    listed = set()
+    for line in open(os.path.join(ROOT, "paper_2207_08393_b200", "csrc", "pairs.def")):
+        m = re.match(r"GLEAM_PAIR\((\d+), (\d+), (\d+), (\d+),", line)
+        if m:
+            listed.add((int(m.group(1)), int(m.group(4)), int(m.group(2))))
+    assert len(listed) >= 300
+    count = 0
+    for n1 in P:
+        for n2 in P:
+            ry = g.gleam_dc_rowtile_split(n1, n2)
+            hit = [t for t in listed if t[0] == n1 and t[1] == n2]
+            assert (ry > 0) == bool(hit), (n1, n2)
+            if hit:
+                assert hit[0][2] == ry and n1 % ry == 0
+                count += 1
+    assert count == len(listed)
+    assert g.gleam_dc_rowtile_split(320, 256) == 16 and g.gleam_dc_rowtile_split(128, 128) > 0
+    assert g.gleam_dc_rowtile_split(640, 256) == 0            # three-stage plan: general middle pass

@@ -67,6 +67,15 @@ def test_rank3_small(oracle, n, mask_kind):
     check(oracle, d, x, y, sens, mask, 1.0, what="rank3 %s kind %d" % (n, mask_kind))
 
 
+@pytest.mark.parametrize("n", [(4, 128, 128), (6, 192, 160), (4, 256, 192), (4, 92, 46), (2, 240, 120), (4, 184, 96), (6, 48, 24)])
+def test_rank3_row_tile_pairs_beyond_the_benchmark_shape(oracle, n):
+    """Extent pairs that used the general strided middle pass before every eligible pair got row-tile kernels."""
+    import paper_2207_08393_b200 as g
+    assert g.gleam_dc_rowtile_split(n[1], n[2]) > 0
+    d, x, y, sens, mask = problem(3, 1, 3, 1, n, MASK_READOUT_INVARIANT, seed=sum(n), density=0.25)
+    check(oracle, d, x, y, sens, mask, 1.0, what="row-tile pair %s" % (n,))
+
+
 def test_rank3_separable_spans_several_chunks(oracle):
     # workspace chunking: 48 MB / (units * n1 * n2 * 8 B) slabs per chunk -> more than one chunk
     d, x, y, sens, mask = problem(3, 1, 8, 1, (12, 320, 256), MASK_READOUT_INVARIANT, seed=5, density=0.1)

@@ -165,6 +165,12 @@ struct SizeImpl {
         }
         return cudaErrorInvalidValue;
     }
+    // The plain strided-axis passes of the full-mask path (no k-space work) run faster on wider tiles (16
+    // neighbouring lines = 128 contiguous bytes per point row; knee3d col_fwd 808 -> 598 us); the pass with the
+    // k-space update measured slower that way (3.4 -> 5.6 ms) and keeps the narrow tile; requesting its mask
+    // weights and measurements before the transform cost registers (104 -> 177, one block less per SM) and
+    // measured slower on volumes as well.
+    static constexpr int LCW = (LC < 16 && sizeof(cf) * (16 * PC::LSZ + 1) <= 100 * 1024 && 16 * PC::MAXBF <= 1024) ? 16 : LC;
     static cudaError_t col(int mode, const ColArgs& a, cudaStream_t s) {
         switch (mode) {
             case COL_Z:        return launch_col<PC, LC, COL_Z>(a, s);
@@ -172,8 +178,8 @@ struct SizeImpl {
                 if constexpr (ColPipe<PC, LC>::ELIGIBLE) return launch_colpipe<PC, LC>(a, s);
                 else return launch_col<PC, LC, COL_MID_SEP>(a, s);
             case COL_MID_FULL: return launch_col<PC, LC, COL_MID_FULL>(a, s);
-            case COL_FWD:      return launch_col<PC, LC, COL_FWD>(a, s);
-            case COL_INV:      return launch_col<PC, LC, COL_INV>(a, s);
+            case COL_FWD:      return launch_col<PC, LCW, COL_FWD>(a, s);
+            case COL_INV:      return launch_col<PC, LCW, COL_INV>(a, s);
             case COL_GRADY:    return launch_col<PC, LC, COL_GRADY>(a, s);
         }
         return cudaErrorInvalidValue;

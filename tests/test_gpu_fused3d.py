@@ -38,6 +38,30 @@ def test_fused_path_matches_oracle(oracle, B, C, T, n):
     assert_close(got_f, ref_f, x, "forward %s" % (n,))
 
 
+def test_fused_path_knee3d_full_size_vjp(oracle):
+    """The whole 320 x 320 x 256 volume with 8 coils through the persistent kernel (320 slabs, 40 turns of the default
+    ring of 8 slabs), element by element against the oracle; the status word stays clear."""
+    import torch
+    import paper_2207_08393_b200 as g
+    from oracle.oracle import Dims
+    from paper_2207_08393_b200 import workloads as wl
+    w = wl.WORKLOADS["knee3d"]
+    inp = wl.make_inputs(w)
+    d = Dims(w.batch, w.coils, w.frames, 3, w.n, 0, MASK_READOUT_INVARIANT)
+    dev = torch.device("cuda:0")
+    tg, ts, tm = (torch.from_numpy(inp[k]).to(dev) for k in ("g", "sens", "mask"))
+    dc = g.DataConsistency(w.batch, w.coils, w.frames, 3, w.n)
+    got = dc.vjp(tg, ts, tm, w.eta)
+    assert g.gleam_dc_check_status(dc.dims()) == 0
+    waits = g.gleam_dc_fused_wait_stats(dc.dims())
+    assert set(waits) == set(g.binding.FUSED_WAIT_KINDS)
+    got = got.cpu().numpy()
+    del tg, ts, tm, dc
+    torch.cuda.empty_cache()
+    ref = oracle.dc_vjp(inp["g"], inp["sens"], inp["mask"], w.eta, d, nthreads=8)
+    assert_close(got, ref, inp["g"], "knee3d vjp through the persistent kernel")
+
+
 def test_fused_path_weighted_mask_in_place_and_per_frame_sens(oracle):
     d, x, y, sens, mask = problem(3, 1, 4, 2, (6, 64, 256), MASK_READOUT_INVARIANT, sens_has_frames=1, weighted=True, seed=3)
     ref = oracle.dc_vjp(x, sens, mask, 1.1, d, nthreads=8)

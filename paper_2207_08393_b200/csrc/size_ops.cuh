@@ -3,6 +3,7 @@
 #pragma once
 #include "dc_kernels.cuh"
 #include "dc_warpline.cuh"
+#include "dc_warpflat.cuh"
 #include "dc_colpipe.cuh"
 
 #include <atomic>
@@ -92,8 +93,35 @@ inline cudaError_t launch_warpline_z(const RowArgs& a, cudaStream_t s) {
                              dim3(WARPS * 32), SMEM, s, a);
 }
 
+// the one-pass kernel with the k-space units numbered across the coils (dc_warpflat.cuh)
+template <class P, bool HAS_Z>
+inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
+    using WF = WarpFlat<P, HAS_Z>;
+    static PerDevice attr_done;
+    static PerDevice slots_cache;
+    cudaError_t e = ensure_smem(warpflat_kernel<P, HAS_Z>, WF::SMEM_BYTES, attr_done);
+    if (e != cudaSuccess) return e;
+    int slots = 0;
+    if ((e = resident_slots(warpflat_kernel<P, HAS_Z>, 32, WF::SMEM_BYTES, slots_cache, &slots)) != cudaSuccess) return e;
+    const long long groups = (a.nrows + WF::LW - 1) / WF::LW;
+    long long blocks = groups;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > slots) blocks = slots;
+    return launch_overlapped(groups <= slots, warpflat_kernel<P, HAS_Z>, dim3((unsigned)blocks), dim3(32), WF::SMEM_BYTES, s, a);
+}
+// GLEAM_NO_FLAT=1 keeps the plain warp-resident kernel for those lengths (tuning aid, read once).
+inline bool flat_enabled() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("GLEAM_NO_FLAT"); v = (e && e[0] == '1') ? 0 : 1; }
+    return v == 1;
+}
+
 template <class P, int MODE>
 inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
+    if constexpr (MODE == ROW_FUSED && WarpFlat<P, false>::ELIGIBLE) {
+        // the numbering across coils pays once a round of 32 units spans more than one coil
+        if (flat_enabled() && a.C >= 2) return a.z != nullptr ? launch_warpflat_z<P, true>(a, s) : launch_warpflat_z<P, false>(a, s);
+    }
     if (MODE == ROW_FUSED && a.z != nullptr) return launch_warpline_z<P, MODE, true>(a, s);
     return launch_warpline_z<P, MODE, false>(a, s);
 }

@@ -19,7 +19,12 @@
 
 namespace gleam {
 
-template <class P, bool HAS_Z>
+#ifdef GLEAM_TRACE
+__device__ long long g_trace[8 * 8192];
+__device__ __forceinline__ long long trace_now() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#endif
+
+template <class P, bool HAS_Z, bool SMW = false>
 struct WarpFlat {
     static constexpr int N = P::N, R0 = P::R0, RL = P::RL;
     static constexpr bool ELIGIBLE = (P::S == 2) && (RL == 8 || RL == 16 || RL == 32) && (R0 < RL) && (N % 2 == 0);
@@ -32,7 +37,7 @@ struct WarpFlat {
         for (int s = SLOTS_MIN; s <= SLOTS_MIN + 3; ++s) if ((s * UPC) % 16 == 0) return s;
         return SLOTS_MIN;
     }
-    static constexpr int SLOTS = (!HAS_Z && slots_aligned() * UPC * USTRIDE * 8 <= 11 * 1024) ? slots_aligned() : SLOTS_MIN;
+    static constexpr int SLOTS = (!SMW && !HAS_Z && slots_aligned() * UPC * USTRIDE * 8 <= 11 * 1024) ? slots_aligned() : SLOTS_MIN;
     static constexpr int ZS = SLOTS + 1;                   // z rows are requested one forward stage ahead
     static constexpr int KCAP = ((N + 3) / 4 + 1) / 2 * 2; // staged z entries per line (more: read from global memory)
     static constexpr int KSTRIDE = KCAP + 2;               // entry KCAP holds zero (unsampled positions point at it)
@@ -44,26 +49,44 @@ struct WarpFlat {
     static constexpr int OFF_K = OFF_IDX + (HAS_Z ? (LW * N + 1) / 2 : 0);
     static constexpr int OFF_CNT = OFF_K + (HAS_Z ? ZS * KTILE : 0);
     static constexpr int ELEMS = (OFF_CNT + (LW + 1) / 2 + 1) / 2 * 2;
-    static constexpr size_t SMEM_BYTES = sizeof(cf) * ELEMS;
+    static constexpr size_t WARP_BYTES = sizeof(cf) * ELEMS;      // per warp of the block
 };
 
-template <class P, bool HAS_Z>
-__global__ void __launch_bounds__(32)
-warpflat_kernel(const RowArgs a) {
+// SMW = false: one warp per block, blocks stride over the line groups.
+// SMW = true (one round, one block per SM, the host sizes the grid): a block of nwhole + 4 nsplit warps.
+// A warp's run time grows with the number of warps on its scheduler (the schedulers favour the oldest warp, and
+// the last one to finish sets the time), so 4 k + 1 single-warp blocks per SM leave one scheduler with k + 1
+// warps and the others waiting for it.  Here the first nwhole warps of the block take one group each, and every
+// further set of four warps (one per scheduler) shares ONE more group, a quarter of the coils each; the partial
+// coil sums are added in warp order through shared memory.  A quarter of the extra work lands on every scheduler.
+// One block per SM also keeps a dependent launch from moving in next to the running one warp by warp, which
+// would fill the schedulers unevenly.
+template <class P, bool HAS_Z, bool SMW>
+__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : 16)
+warpflat_kernel(const RowArgs a, const int nwhole) {
     grid_dependency_wait();
     grid_launch_dependents();
-    using WF = WarpFlat<P, HAS_Z>;
+#ifdef GLEAM_TRACE
+    const long long tr_t0 = trace_now();
+    long long tr_t1 = 0;
+#endif
+    using WF = WarpFlat<P, HAS_Z, SMW>;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL, LW = WF::LW, UPC = WF::UPC, US = WF::USTRIDE, SLOTS = WF::SLOTS;
     constexpr int KCAP = WF::KCAP, KSTRIDE = WF::KSTRIDE, KTILE = WF::KTILE, ZS = WF::ZS, MS = WF::MS;
     extern __shared__ __align__(16) float2 smem[];
-    cf* sX = smem + WF::OFF_X;
-    cf* sE = smem + WF::OFF_E;
-    float* sM = reinterpret_cast<float*>(smem + WF::OFF_M2);
-    int* sI = reinterpret_cast<int*>(smem + WF::OFF_IDX);
-    cf* sK = smem + WF::OFF_K;
-    int* sC = reinterpret_cast<int*>(smem + WF::OFF_CNT);    // per line: sampled entries, -1 for a line past the end
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    cf* wsm = smem + warp * WF::ELEMS;
+    cf* sX = wsm + WF::OFF_X;
+    cf* sE = wsm + WF::OFF_E;
+    float* sM = reinterpret_cast<float*>(wsm + WF::OFF_M2);
+    int* sI = reinterpret_cast<int*>(wsm + WF::OFF_IDX);
+    cf* sK = wsm + WF::OFF_K;
+    int* sC = reinterpret_cast<int*>(wsm + WF::OFF_CNT);    // per line: sampled entries, -1 for a line past the end
+    const bool split = SMW && warp >= nwhole;                      // one of four warps that share a group
+    const int set = split ? (warp - nwhole) >> 2 : 0, q = split ? (warp - nwhole) & 3 : 0;
+    const int cbase = split ? q * a.C / 4 : 0;                     // first coil and number of coils of this warp
+    const int nc = split ? (q + 1) * a.C / 4 - cbase : a.C;
 
-    const int lane = threadIdx.x;
     const int l = lane / RL, j = lane % RL;                 // image-side identity: line of the warp, butterfly
 
     cf tw0[R0];
@@ -75,9 +98,12 @@ warpflat_kernel(const RowArgs a) {
         __syncwarp();
     }
     const long long ngroups = (a.nrows + LW - 1) / LW;
-    const int total = UPC * a.C, rounds = (total + 31) / 32;
+    const int total = UPC * nc, rounds = (total + 31) / 32;
+    const long long g_first = !SMW ? (long long)blockIdx.x
+                            : split ? (long long)(nwhole + set) * gridDim.x + blockIdx.x : (long long)warp * gridDim.x + blockIdx.x;
+    const long long g_step = !SMW ? (long long)gridDim.x : ngroups;              // SMW: a single round
 
-    for (long long g = blockIdx.x; g < ngroups; g += gridDim.x) {
+    for (long long g = g_first; g < ngroups; g += g_step) {
         const long long row = g * LW + l;
         const bool row_ok = row < a.nrows;
         const unsigned rowu = row_ok ? (unsigned)row : 0u;       // host side guarantees nrows < 2^31
@@ -85,8 +111,9 @@ warpflat_kernel(const RowArgs a) {
         const int ri = (int)(rowu - bt * (unsigned)a.rpb);
         const int b = (int)(bt / (unsigned)a.T), t = (int)(bt - (unsigned)b * (unsigned)a.T);
         const long long x_off = ((long long)bt * a.RPB + a.row0 + ri) * N;
-        const long long s_off = (((long long)(b * a.C) * a.Ts + (a.Ts > 1 ? t : 0)) * a.RPB + a.row0 + ri) * N;
-        const long long k_off = (((long long)(b * a.C) * a.T + t) * a.RPB + a.row0 + ri) * N;
+        // coil indices below are relative to cbase
+        const long long s_off = (((long long)(b * a.C + cbase) * a.Ts + (a.Ts > 1 ? t : 0)) * a.RPB + a.row0 + ri) * N;
+        const long long k_off = (((long long)(b * a.C + cbase) * a.T + t) * a.RPB + a.row0 + ri) * N;
         const long long s_stride = (long long)a.Ts * a.RPB * N;
         const long long k_stride = (long long)a.T * a.RPB * N;
         const cf* sp = a.sens + s_off + j;                       // this lane's sensitivities of coil 0
@@ -156,21 +183,24 @@ warpflat_kernel(const RowArgs a) {
 #pragma unroll
         for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
         cf sf[R0];                       // sensitivities of the next forward image-side stage
-        load_sens(sf, 0);
+        if (nc > 0) load_sens(sf, 0);
+#ifdef GLEAM_TRACE
+        tr_t1 = trace_now();
+#endif
         int af = 0, ai = 0;              // next coil of the forward / of the inverse image-side stage
 
         for (int br = 0; br < rounds; ++br) {
             const int upto = min(32 * (br + 1), total);
             const int need = (upto + UPC - 1) / UPC;                     // coils this round draws units from
-            const int done = (br == rounds - 1) ? a.C : upto / UPC;      // coils complete after this round
+            const int done = (br == rounds - 1) ? nc : upto / UPC;       // coils complete after this round
             // ---- forward image-side stage: S x, R0-point butterflies, twiddles, into the ring ----
             while (af < need) {
-                if (HAS_Z) { if (af + 1 < a.C) issue_z(af + 1); cp_async_commit(); }
+                if (HAS_Z) { if (af + 1 < nc) issue_z(af + 1); cp_async_commit(); }
                 if (af == 0) { cp_async_wait<HAS_Z ? 1 : 0>(); __syncwarp(); }      // x (and z of coil 0) have landed
                 cf v[R0];
 #pragma unroll
                 for (int m = 0; m < R0; ++m) v[m] = cmul(sf[m], x_at(j + RL * m));
-                if (af + 1 < a.C) load_sens(sf, af + 1);
+                if (af + 1 < nc) load_sens(sf, af + 1);
                 Dft<R0, -1>::run(v);
                 cf* e = sE + ((af % SLOTS) * UPC + l * R0) * US + j;
 #pragma unroll
@@ -247,6 +277,21 @@ warpflat_kernel(const RowArgs a) {
             }
         }
         cp_async_wait<0>();
+        __syncwarp();
+        if (SMW && split) {
+            // partial coil sums of the other three warps are added by the first in warp order (the ring is free by now)
+            if (q > 0) {
+#pragma unroll
+                for (int m = 0; m < R0; ++m) sE[m * 32 + lane] = acc[m];
+            }
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + set) : "memory");      // the four warps of this group (every one gets here: same g)
+            if (q > 0) continue;
+            for (int w = 1; w < 4; ++w) {
+                const cf* o = smem + (nwhole + 4 * set + w) * WF::ELEMS + WF::OFF_E;
+#pragma unroll
+                for (int m = 0; m < R0; ++m) acc[m] = cadd(acc[m], o[m * 32 + lane]);
+            }
+        }
         // ---- out = x - eta * sum, and Re<x, out> per row for the caller's inner product ----
         double dsum = 0.0;
         if (row_ok) {
@@ -263,6 +308,14 @@ warpflat_kernel(const RowArgs a) {
             if (j == 0 && row_ok) a.dot_rows[row] = dsum;
         }
     }
+#ifdef GLEAM_TRACE
+    if ((threadIdx.x & 31) == 0) {
+        unsigned sm_, w_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); asm volatile("mov.u32 %0, %%warpid;" : "=r"(w_));
+        const int slot = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) & 8191;
+        g_trace[8 * slot + 0] = tr_t0; g_trace[8 * slot + 1] = tr_t1; g_trace[8 * slot + 2] = trace_now();
+        g_trace[8 * slot + 3] = sm_; g_trace[8 * slot + 4] = w_; g_trace[8 * slot + 5] = blockIdx.x; g_trace[8 * slot + 6] = threadIdx.x >> 5;
+    }
+#endif
 }
 
 }  // namespace gleam

@@ -93,21 +93,49 @@ inline cudaError_t launch_warpline_z(const RowArgs& a, cudaStream_t s) {
                              dim3(WARPS * 32), SMEM, s, a);
 }
 
+// GLEAM_NO_SPLIT=1 keeps single-warp blocks for every group (tuning aid, read once).
+inline bool split_enabled() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("GLEAM_NO_SPLIT"); v = (e && e[0] == '1') ? 0 : 1; }
+    return v == 1;
+}
+
 // the one-pass kernel with the k-space units numbered across the coils (dc_warpflat.cuh)
 template <class P, bool HAS_Z>
 inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
-    using WF = WarpFlat<P, HAS_Z>;
+    using WF = WarpFlat<P, HAS_Z, false>;
     static PerDevice attr_done;
     static PerDevice slots_cache;
-    cudaError_t e = ensure_smem(warpflat_kernel<P, HAS_Z>, WF::SMEM_BYTES, attr_done);
+    cudaError_t e = ensure_smem(warpflat_kernel<P, HAS_Z, false>, WF::WARP_BYTES, attr_done);
     if (e != cudaSuccess) return e;
     int slots = 0;
-    if ((e = resident_slots(warpflat_kernel<P, HAS_Z>, 32, WF::SMEM_BYTES, slots_cache, &slots)) != cudaSuccess) return e;
+    if ((e = resident_slots(warpflat_kernel<P, HAS_Z, false>, 32, WF::WARP_BYTES, slots_cache, &slots)) != cudaSuccess) return e;
     const long long groups = (a.nrows + WF::LW - 1) / WF::LW;
+    if (groups <= 0) return cudaSuccess;
+    // One round of 8 to 16 groups per SM: one block per SM that holds all its warps.  4 k + 1 (or 4 k + 2) groups per
+    // SM: the groups beyond 4 k are split by coils over four warps each, one per scheduler.  (Measured on cine-shaped
+    // problems, per call: 13 groups per SM 18.7 -> 16.6 us, 12 per SM 18.7 -> 15.3 us; up to 7 per SM single-warp
+    // blocks are faster, 11.3 against 12.7 us.)
+    if constexpr (!HAS_Z) {
+        using WS = WarpFlat<P, HAS_Z, true>;
+        static PerDevice attrs_done;
+        int sms = 0, dev = 0;
+        if (split_enabled() && groups <= slots && cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0 && groups > 7LL * sms) {
+            const int per = (int)((groups + sms - 1) / sms);
+            int nsplit = (a.C >= 4 && (per % 4 == 1 || per % 4 == 2)) ? per % 4 : 0;
+            if (per - nsplit + 4 * nsplit > 16) nsplit = 0;
+            const int nwhole = per - nsplit, warps = nwhole + 4 * nsplit;
+            const size_t bytes = WS::WARP_BYTES * (size_t)warps;
+            if (warps <= 16 && bytes <= 227 * 1024) {
+                if ((e = ensure_smem(warpflat_kernel<P, HAS_Z, true>, 16 * WS::WARP_BYTES, attrs_done)) != cudaSuccess) return e;
+                return launch_overlapped(true, warpflat_kernel<P, HAS_Z, true>, dim3((unsigned)sms), dim3(32 * warps), bytes, s, a, nwhole);
+            }
+        }
+    }
     long long blocks = groups;
-    if (blocks <= 0) return cudaSuccess;
     if (blocks > slots) blocks = slots;
-    return launch_overlapped(groups <= slots, warpflat_kernel<P, HAS_Z>, dim3((unsigned)blocks), dim3(32), WF::SMEM_BYTES, s, a);
+    return launch_overlapped(groups <= slots, warpflat_kernel<P, HAS_Z, false>, dim3((unsigned)blocks), dim3(32), WF::WARP_BYTES, s, a, 1);
 }
 // GLEAM_NO_FLAT=1 keeps the plain warp-resident kernel for those lengths (tuning aid, read once).
 inline bool flat_enabled() {

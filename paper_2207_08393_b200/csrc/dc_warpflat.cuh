@@ -38,17 +38,19 @@ struct WarpFlat {
         return SLOTS_MIN;
     }
     static constexpr int SLOTS = (!SMW && !HAS_Z && slots_aligned() * UPC * USTRIDE * 8 <= 11 * 1024) ? slots_aligned() : SLOTS_MIN;
-    static constexpr int ZS = SLOTS + 1;                   // z rows are requested one forward stage ahead
+    static constexpr int ZS = SMW ? SLOTS : SLOTS + 1;     // z rows are requested one forward stage ahead (SMW: in their own stage)
     static constexpr int KCAP = ((N + 3) / 4 + 1) / 2 * 2; // staged z entries per line (more: read from global memory)
     static constexpr int KSTRIDE = KCAP + 2;               // entry KCAP holds zero (unsampled positions point at it)
     static constexpr int KTILE = LW * KSTRIDE;
     static constexpr int MS = N + ((LW > 1 && N % 32 == 0) ? 16 : 0);   // mask row stride (floats): lines on different banks
     // shared memory of the warp, in float2 units
     static constexpr int OFF_X = 0, OFF_E = LW * N, OFF_M2 = OFF_E + SLOTS * UPC * USTRIDE + (SLOTS * UPC * USTRIDE) % 2;
-    static constexpr int OFF_IDX = OFF_M2 + (LW * MS + 1) / 2;
-    static constexpr int OFF_K = OFF_IDX + (HAS_Z ? (LW * N + 1) / 2 : 0);
+    // mask weights: one float per raw k (no z), or one per sampled rank next to 16-bit ranks of every raw k (with z)
+    static constexpr int OFF_IDX = OFF_M2 + ((HAS_Z ? LW * KSTRIDE : LW * MS) + 3) / 4 * 2;
+    static constexpr int OFF_K = OFF_IDX + (HAS_Z ? (LW * N + 7) / 8 * 2 : 0);
     static constexpr int OFF_CNT = OFF_K + (HAS_Z ? ZS * KTILE : 0);
-    static constexpr int ELEMS = (OFF_CNT + (LW + 1) / 2 + 1) / 2 * 2;
+    // per line: element offset of its z row (64-bit), sampled count, mask row index
+    static constexpr int ELEMS = (OFF_CNT + 2 * LW + 1) / 2 * 2;
     static constexpr size_t WARP_BYTES = sizeof(cf) * ELEMS;      // per warp of the block
 };
 
@@ -79,9 +81,11 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
     cf* sX = wsm + WF::OFF_X;
     cf* sE = wsm + WF::OFF_E;
     float* sM = reinterpret_cast<float*>(wsm + WF::OFF_M2);
-    int* sI = reinterpret_cast<int*>(wsm + WF::OFF_IDX);
+    short* sI = reinterpret_cast<short*>(wsm + WF::OFF_IDX);
     cf* sK = wsm + WF::OFF_K;
-    int* sC = reinterpret_cast<int*>(wsm + WF::OFF_CNT);    // per line: sampled entries, -1 for a line past the end
+    long long* sKo = reinterpret_cast<long long*>(wsm + WF::OFF_CNT);      // per line: offset of the z row of coil cbase
+    int* sC = reinterpret_cast<int*>(wsm + WF::OFF_CNT + LW);              // per line: sampled entries, -1 for a line past the end
+    unsigned* sBt = reinterpret_cast<unsigned*>(sC + LW);                   // per line: mask row
     const bool split = SMW && warp >= nwhole;                      // one of four warps that share a group
     const int set = split ? (warp - nwhole) >> 2 : 0, q = split ? (warp - nwhole) & 3 : 0;
     const int cbase = split ? q * a.C / 4 : 0;                     // first coil and number of coils of this warp
@@ -89,14 +93,16 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 
     const int l = lane / RL, j = lane % RL;                 // image-side identity: line of the warp, butterfly
 
+    if (HAS_Z) {
+        for (int i = lane; i < ZS * LW; i += 32) sK[(i / LW) * KTILE + (i % LW) * KSTRIDE + KCAP] = make_float2(0.f, 0.f);
+        if (lane < LW) sM[lane * KSTRIDE + KCAP] = 0.f;
+        __syncwarp();
+    }
+    // inter-stage twiddles exp(-2 pi i j k / N) of this lane (fetching them again before the image-side stages of
+    // every round, to free registers for the k-space round, was measured slower: 18.7 against 16.4 us per call)
     cf tw0[R0];
 #pragma unroll
     for (int k = 0; k < R0; ++k) tw0[k] = unit_root_fwd<N>((j * k) % N);
-
-    if (HAS_Z) {
-        for (int i = lane; i < ZS * LW; i += 32) sK[(i / LW) * KTILE + (i % LW) * KSTRIDE + KCAP] = make_float2(0.f, 0.f);
-        __syncwarp();
-    }
     const long long ngroups = (a.nrows + LW - 1) / LW;
     const int total = UPC * nc, rounds = (total + 31) / 32;
     const long long g_first = !SMW ? (long long)blockIdx.x
@@ -142,28 +148,33 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
             for (int k0 = 0; k0 < N; k0 += 32) {
                 const int k = k0 + lane;
                 const float mv = (k < N) ? a.mask[bto * N + shift_half(k, N)] : 0.f;
-                if (k < N) sM[ll * MS + k] = mv * mv * (1.0f / N);
-                if (HAS_Z) {
+                if (!HAS_Z) {
+                    if (k < N) sM[ll * MS + k] = mv * mv * (1.0f / N);
+                } else {
                     const unsigned bal = __ballot_sync(0xffffffffu, mv != 0.f);
-                    if (k < N) sI[ll * N + k] = (mv != 0.f) ? cnt + __popc(bal & ((1u << lane) - 1u)) : -1;
+                    const int r = cnt + __popc(bal & ((1u << lane) - 1u));
+                    if (k < N) sI[ll * N + k] = (short)((mv != 0.f) ? r : -1);
+                    if (mv != 0.f && r < KCAP) sM[ll * KSTRIDE + r] = mv * mv * (1.0f / N);
                     cnt += __popc(bal);
                 }
             }
             if (lane == 0) sC[ll] = cnt;
+            if (HAS_Z && lane == ll * RL) { sKo[ll] = k_off; sBt[ll] = bt; }
         }
         __syncwarp();
         // z row of coil c for every line of the warp -> slot c % ZS
         auto issue_z = [&](int c) {
 #pragma unroll
             for (int ll = 0; ll < LW; ++ll) {
-                const long long ko = __shfl_sync(0xffffffffu, k_off, ll * RL);
+                const long long ko = sKo[ll];
                 const int kc = sC[ll];
                 if (kc <= 0 || kc > KCAP) continue;
                 const cf* ks = a.z + ko + c * k_stride;
                 for (int i = lane; i < (kc + 1) / 2; i += 32) cp_async16(sK + (c % ZS) * KTILE + ll * KSTRIDE + 2 * i, ks + 2 * i);
             }
         };
-        if (HAS_Z) issue_z(0);
+        constexpr int ZAHEAD = SMW ? 0 : 1;      // forward stages between the request for a z row and the stage of its coil
+        if (HAS_Z && ZAHEAD) issue_z(0);
         cp_async_commit();
 
         const bool x_planes = a.x_planar && (N % 4 == 0);          // x staged as two planes of floats
@@ -195,7 +206,7 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
             const int done = (br == rounds - 1) ? nc : upto / UPC;       // coils complete after this round
             // ---- forward image-side stage: S x, R0-point butterflies, twiddles, into the ring ----
             while (af < need) {
-                if (HAS_Z) { if (af + 1 < nc) issue_z(af + 1); cp_async_commit(); }
+                if (HAS_Z) { if (af + ZAHEAD < nc) issue_z(af + ZAHEAD); cp_async_commit(); }
                 if (af == 0) { cp_async_wait<HAS_Z ? 1 : 0>(); __syncwarp(); }      // x (and z of coil 0) have landed
                 cf v[R0];
 #pragma unroll
@@ -207,7 +218,7 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
                 for (int k = 0; k < R0; ++k) e[k * US] = (k == 0) ? v[0] : cmul(v[k], tw0[k]);
                 ++af;
             }
-            if (HAS_Z) cp_async_wait<1>();       // everything but the newest request (the next coil's z) is there
+            if (HAS_Z) cp_async_wait<ZAHEAD>();  // everything but a request for the next coil's z is there
             __syncwarp();
             // ---- k-space round: units 32 br .. 32 br + 31, one per lane ----
             {
@@ -221,32 +232,44 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 #pragma unroll
                 for (int m = 0; m < RL; ++m) u[m] = e[m];
                 Dft<RL, -1>::run(u);
-                const float* mm = sM + bl * MS + jb;
-                const int kc = HAS_Z ? sC[bl] : 0;
-                const long long kob = HAS_Z ? __shfl_sync(0xffffffffu, k_off, bl * RL) : 0;   // z row of the unit's line
-                if (HAS_Z && kc > 0 && kc <= KCAP) {
-                    // staged z: unsampled entries read the zero slot
-                    const int* ri_ = sI + bl * N + jb;
-                    const cf* zk = sK + (c % ZS) * KTILE + bl * KSTRIDE;
+                if (!HAS_Z) {
+                    const float* mm = sM + bl * MS + jb;
 #pragma unroll
-                    for (int k = 0; k < RL; ++k) {
-                        const float wv = mm[R0 * k];
-                        const int r = ri_[R0 * k];
-                        const cf q = zk[(r >= 0) ? r : KCAP];
-                        u[k] = make_float2(fmaf(wv, u[k].x, -q.x), fmaf(wv, u[k].y, -q.y));
-                    }
+                    for (int k = 0; k < RL; ++k) u[k] = cscale(u[k], mm[R0 * k]);
                 } else {
+                    const int kc = sC[bl];
+                    const short* ri_ = sI + bl * N + jb;
+                    if (kc > 0 && kc <= KCAP) {
+                        // staged z and weights by rank: unsampled entries read the zero slots
+                        const float* mw = sM + bl * KSTRIDE;
+                        const cf* zk = sK + (c % ZS) * KTILE + bl * KSTRIDE;
 #pragma unroll
-                    for (int k = 0; k < RL; ++k) {
-                        const float wv = mm[R0 * k];
-                        u[k] = cscale(u[k], wv);
-                        if (HAS_Z && kc > KCAP) {   // more sampled entries than the stage holds: from global memory
-                            const int r = sI[bl * N + jb + R0 * k];
-                            if (r >= 0 && r < N) {
-                                const cf q = a.z[kob + c * k_stride + r];
+                        for (int k = 0; k < RL; ++k) {
+                            const int r = ri_[R0 * k];
+                            const int rr = (r >= 0) ? r : KCAP;
+                            const float wv = mw[rr];
+                            const cf q = zk[rr];
+                            u[k] = make_float2(fmaf(wv, u[k].x, -q.x), fmaf(wv, u[k].y, -q.y));
+                            if (k % 4 == 3) asm volatile("" ::: "memory");     // four entries in flight at a time: registers
+                        }
+                    } else if (kc > KCAP) {
+                        // more sampled entries than the stage holds: weights and z from global memory
+                        const float* mrow = a.mask + (long long)sBt[bl] * N;
+                        const cf* zrow = a.z + sKo[bl] + c * k_stride;
+#pragma unroll
+                        for (int k = 0; k < RL; ++k) {
+                            const float mv = mrow[shift_half(jb + R0 * k, N)];
+                            u[k] = cscale(u[k], mv * mv * (1.0f / N));
+                            const int r = ri_[R0 * k];
+                            if (r >= 0) {
+                                const cf q = zrow[r];
                                 u[k] = make_float2(u[k].x - q.x, u[k].y - q.y);
                             }
+                            asm volatile("" ::: "memory");      // one entry at a time: this rare path must not cost registers
                         }
+                    } else {       // nothing sampled on this line (or no line)
+#pragma unroll
+                        for (int k = 0; k < RL; ++k) u[k] = make_float2(0.f, 0.f);
                     }
                 }
                 Dft<RL, +1>::run(u);
@@ -284,7 +307,8 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 #pragma unroll
                 for (int m = 0; m < R0; ++m) sE[m * 32 + lane] = acc[m];
             }
-            asm volatile("bar.sync %0, 128;" ::"r"(1 + set) : "memory");      // the four warps of this group (every one gets here: same g)
+            // the four warps of this group (every one gets here: same g)
+            if (set == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
             if (q > 0) continue;
             for (int w = 1; w < 4; ++w) {
                 const cf* o = smem + (nwhole + 4 * set + w) * WF::ELEMS + WF::OFF_E;

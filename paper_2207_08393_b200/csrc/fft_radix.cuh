@@ -4,7 +4,8 @@
 //     X[k] = sum_n x[n] * exp(DIR * 2 pi i * n k / R),   DIR = -1 (forward) or +1 (inverse),
 // in place on a register array, natural order in and out.  Radices: 2 and 4 are written out,
 // odd primes use the symmetric direct form (pairs x[m] +- x[R-m], real cosine / sine sums),
-// composites are split Cooley-Tukey style with the inner twiddles folded in as constants.
+// composites with coprime factors use the prime-factor index maps (no inner twiddles), the others
+// are split Cooley-Tukey style with the inner twiddles folded in as constants.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -216,9 +217,41 @@ template <int R, int DIR> struct DftComposite {
     }
 };
 
+// composite R = A * B with coprime factors (6, 10, 12, 15, 20, ...): prime-factor index maps,
+//   n = (B n1 + A n2) mod R,   k = the residue with k mod A = k1 and k mod B = k2,
+// turn the transform into A-point and B-point transforms with no twiddle factors in between
+// (W_R^{B n1 k} = W_A^{n1 k1},  W_R^{A n2 k} = W_B^{n2 k2}).
+constexpr int ct_gcd(int a, int b) { return b == 0 ? a : ct_gcd(b, a % b); }
+constexpr int crt_index(int k1, int A, int k2, int B) {
+    for (int k = 0; k < A * B; ++k) if (k % A == k1 && k % B == k2) return k;
+    return 0;
+}
+template <int R, int DIR> struct DftCoprime {
+    static constexpr int A = ct_factor(R);
+    static constexpr int B = R / A;
+    static GLEAM_HD void run(cf (&v)[R]) {
+        cf y[A][B];
+        static_for<0, A>([&](auto n1i) {
+            constexpr int n1 = decltype(n1i)::value;
+            cf t[B];
+            static_for<0, B>([&](auto n2i) { constexpr int n2 = decltype(n2i)::value; t[n2] = v[(B * n1 + A * n2) % R]; });
+            Dft<B, DIR>::run(t);
+            static_for<0, B>([&](auto k2i) { constexpr int k2 = decltype(k2i)::value; y[n1][k2] = t[k2]; });
+        });
+        static_for<0, B>([&](auto k2i) {
+            constexpr int k2 = decltype(k2i)::value;
+            cf t[A];
+            static_for<0, A>([&](auto n1i) { constexpr int n1 = decltype(n1i)::value; t[n1] = y[n1][k2]; });
+            Dft<A, DIR>::run(t);
+            static_for<0, A>([&](auto k1i) { constexpr int k1 = decltype(k1i)::value; v[crt_index(k1, A, k2, B)] = t[k1]; });
+        });
+    }
+};
+
 template <int R, int DIR> struct Dft {
     static GLEAM_HD void run(cf (&v)[R]) {
         if constexpr (R % 2 == 1 && smallest_odd_factor(R) == R) DftPrime<R, DIR>::run(v);
+        else if constexpr (ct_gcd(ct_factor(R), R / ct_factor(R)) == 1) DftCoprime<R, DIR>::run(v);
         else DftComposite<R, DIR>::run(v);
     }
 };

@@ -116,7 +116,7 @@ inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
     // SM: the groups beyond 4 k are split by coils over four warps each, one per scheduler.  (Measured on cine-shaped
     // problems, per call: 13 groups per SM 18.7 -> 16.6 us, 12 per SM 18.7 -> 15.3 us; up to 7 per SM single-warp
     // blocks are faster, 11.3 against 12.7 us.)
-    if constexpr (!HAS_Z) {
+    {
         using WS = WarpFlat<P, HAS_Z, true>;
         static PerDevice attrs_done;
         int sms = 0, dev = 0;
@@ -127,7 +127,9 @@ inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
             if (per - nsplit + 4 * nsplit > 16) nsplit = 0;
             const int nwhole = per - nsplit, warps = nwhole + 4 * nsplit;
             const size_t bytes = WS::WARP_BYTES * (size_t)warps;
-            if (warps <= 16 && bytes <= 227 * 1024) {
+            // with z the split groups were measured slower than single-warp blocks (13 groups per SM: 25.2 against
+            // 24.7 us per call), whole groups alone faster (12 per SM: 22.5 against 24.5 us)
+            if (warps <= 16 && bytes <= 227 * 1024 && !(HAS_Z && nsplit > 0)) {
                 if ((e = ensure_smem(warpflat_kernel<P, HAS_Z, true>, 16 * WS::WARP_BYTES, attrs_done)) != cudaSuccess) return e;
                 return launch_overlapped(true, warpflat_kernel<P, HAS_Z, true>, dim3((unsigned)sms), dim3(32 * warps), bytes, s, a, nwhole);
             }

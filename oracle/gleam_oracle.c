@@ -553,6 +553,31 @@ int oracle_modl_cg_vjp(const float* g, const float* sens, const float* mask, dou
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Eq. 3 in its normal-equations form.  A^H (A x - y) = A^H A x - A^H y, so with the zero-filled
+ * image  aty = A^H y  given (it does not change over the unrolled iterations of one example)
+ *
+ *      out = x - eta * (A^H A x - aty).
+ *
+ * aty: (B, T, n0, n1, n2) single-precision complex, as the GPU call receives it.  Steps: the
+ * vector-Jacobian form of oracle_dc gives x - eta A^H A x; eta * aty is added to it.
+ * Pins (tests/test_oracle_aty.py): dense-matrix brute force, equality with oracle_dc for
+ * aty = A^H y, aty = 0 gives the vector-Jacobian product, exact linearity in aty.
+ * ------------------------------------------------------------------------------------------ */
+int oracle_dc_aty(const float* x, const float* aty, const float* sens, const float* mask, double eta,
+                  const int64_t* dims, zc* out, int nthreads)
+{
+    odims o;
+    if (parse_dims(dims, &o) != ORACLE_OK) return ORACLE_ERR_ARG;
+    if (!x || !aty || !sens || !mask || !out) return ORACLE_ERR_ARG;
+    const int rc = oracle_dc(x, NULL, sens, mask, eta, dims, out, nthreads);
+    if (rc != ORACLE_OK) return rc;
+    const int64_t total = o.B * o.T * o.V;
+    for (int64_t p = 0; p < total; ++p)
+        out[p] += eta * ((double)aty[2 * p] + I * (double)aty[2 * p + 1]);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Gradients of the data-consistency step (Eq. 3) with respect to its two other inputs, for a
  * cotangent g of the output (conjugate-Wirtinger convention, as for the vector-Jacobian product
  * with respect to x).  out = x - eta A^H (A x - y) is linear in eta and affine in y, so both are

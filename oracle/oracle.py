@@ -52,6 +52,8 @@ def _load():
         lib.oracle_apply_AH.restype = i32
         lib.oracle_dc.argtypes = [p, p, p, p, dbl, p, p, i32]
         lib.oracle_dc.restype = i32
+        lib.oracle_dc_aty.argtypes = [p, p, p, p, dbl, p, p, i32]
+        lib.oracle_dc_aty.restype = i32
         lib.oracle_modl_cg.argtypes = [p, p, p, p, dbl, i32, p, p, i32]
         lib.oracle_modl_cg.restype = i32
         lib.oracle_modl_cg_vjp.argtypes = [p, p, p, dbl, i32, p, p, i32]
@@ -202,6 +204,17 @@ def dc_forward(x, y, sens, mask, eta: float, d: Dims, nthreads: int = 1) -> np.n
     out = np.empty(d.image_shape(), dtype=np.complex128)
     dd = d.as_array()
     rc = _load().oracle_dc(_ptr(x), _ptr(y), _ptr(sens), _ptr(mask), float(eta), _ptr(dd), _ptr(out), nthreads)
+    assert rc == 0, rc
+    return out
+
+
+def dc_forward_aty(x, aty, sens, mask, eta: float, d: Dims, nthreads: int = 1) -> np.ndarray:
+    """Eq. 3 in normal-equations form: out = x - eta (A^H A x - aty), aty = A^H y given as complex64."""
+    x = _c64(x, d.image_shape()); aty = _c64(aty, d.image_shape())
+    sens = _c64(sens, d.sens_shape()); mask = _f32(mask, d.mask_shape())
+    out = np.empty(d.image_shape(), dtype=np.complex128)
+    dd = d.as_array()
+    rc = _load().oracle_dc_aty(_ptr(x), _ptr(aty), _ptr(sens), _ptr(mask), float(eta), _ptr(dd), _ptr(out), nthreads)
     assert rc == 0, rc
     return out
 

@@ -221,6 +221,24 @@ GLEAM_API int gleam_dc_prepare(const void* y, const float* mask, const gleam_dim
 GLEAM_API int gleam_dc_forward_prepared(const void* x, const void* y, const void* sens, const float* mask,
                                         float eta, void* out, const gleam_dims* dims);
 
+/* ---- the step in its normal-equations form ----------------------------------------------------
+ * A^H (A x - y) = A^H A x - A^H y, so Eq. 3 is also
+ *
+ *      out = x - eta * (A^H A x - aty),        aty = A^H y   (gleam_dc_adjoint),
+ *
+ * and the zero-filled image A^H y of an example is the same for all unrolled iterations and all
+ * greedy modules of Alg. 1 (it is the usual starting image x^0 as well).  With it given, a step
+ * costs what gleam_dc_vjp costs: no pass over y, no table of y, no per-sample look-up.
+ *   aty : device, complex64, (B, T, n0, n1, n2), 16-byte aligned; may alias x, must not overlap out
+ *         or the workspace.  Any image is accepted (the call evaluates the formula above).
+ * Other arguments, workspace (that of gleam_dc_vjp), in-place rule (out == x allowed) and errors
+ * as for gleam_dc_forward.  The vector-Jacobian product with respect to x is gleam_dc_vjp; the
+ * cotangent of aty is eta * grad_out.  The result equals gleam_dc_forward(x, y, ...) up to
+ * single-precision rounding (different order of operations), not bit for bit.
+ */
+GLEAM_API int gleam_dc_forward_aty(const void* x, const void* aty, const void* sens, const float* mask, float eta,
+                                   void* out, const gleam_dims* dims);
+
 /* ---- zero-filled SENSE image -----------------------------------------------------------------
  * out = A^H y = sum_c conj(S_c) F^H (Omega y_c): the image the paper's networks start from (its
  * Experiments section feeds "zero-filled, SENSE-reconstructed" images).  Evaluated as Eq. 3 on a

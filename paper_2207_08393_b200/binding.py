@@ -35,7 +35,7 @@ EXPORTS = ["gleam_dc_forward", "gleam_dc_vjp", "gleam_dc_workspace_size", "gleam
            "gleam_dc_host_arena_size", "gleam_dc_launch_count", "gleam_dc_profile_begin", "gleam_dc_profile_end",
            "gleam_dc_forward_static", "gleam_dc_static_scratch_bytes",
            "gleam_modl_cg_forward", "gleam_modl_cg_vjp", "gleam_modl_cg_workspace_size",
-           "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_adjoint",
+           "gleam_dc_prepare", "gleam_dc_forward_prepared", "gleam_dc_forward_aty", "gleam_dc_adjoint",
            "gleam_dc_check_status", "gleam_dc_debug_fused", "gleam_dc_fused_wait_stats", "gleam_dc_set_fused",
            "gleam_dc_grad_eta", "gleam_dc_grad_y", "gleam_dc_grad_workspace_size",
            "gleam_dc_forward_layout", "gleam_dc_vjp_layout", "gleam_l1_loss", "gleam_l1_loss_workspace_size",
@@ -110,6 +110,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         lib.gleam_dc_prepare.restype = i32
         lib.gleam_dc_forward_prepared.argtypes = [vp, vp, vp, vp, f32, vp, dp]
         lib.gleam_dc_forward_prepared.restype = i32
+        lib.gleam_dc_forward_aty.argtypes = [vp, vp, vp, vp, f32, vp, dp]
+        lib.gleam_dc_forward_aty.restype = i32
         lib.gleam_modl_cg_forward.argtypes = [vp, vp, vp, vp, f32, ctypes.c_int32, vp, dp]
         lib.gleam_modl_cg_forward.restype = i32
         lib.gleam_modl_cg_vjp.argtypes = [vp, vp, vp, f32, ctypes.c_int32, vp, dp]
@@ -225,6 +227,12 @@ def gleam_dc_prepare(y, mask, dims: gleam_dims) -> None:
     """Computes what Eq. 3 needs from y and the mask alone into dims.workspace (kept by the caller
     until the last gleam_dc_forward_prepared)."""
     _check(load_library().gleam_dc_prepare(_addr(y), _addr(mask), ctypes.byref(dims)))
+
+
+def gleam_dc_forward_aty(x, aty, sens, mask, eta, out, dims: gleam_dims) -> None:
+    """Eq. 3 in normal-equations form: out = x - eta (A^H A x - aty) with aty = A^H y given as an image."""
+    _check(load_library().gleam_dc_forward_aty(_addr(x), _addr(aty), _addr(sens), _addr(mask), float(eta),
+                                               _addr(out), ctypes.byref(dims)))
 
 
 def gleam_dc_forward_prepared(x, y, sens, mask, eta, out, dims: gleam_dims) -> None:
@@ -405,6 +413,13 @@ class DataConsistency:
         """For unrolled iterations with the same y and mask: fills the workspace once; follow with
         forward_prepared calls only (forward and vjp of this object would overwrite it)."""
         gleam_dc_prepare(y, mask, self.dims())
+
+    def forward_aty(self, x, aty, sens, mask, eta, out=None):
+        """The step with the zero-filled image aty = A^H y (``adjoint``) given instead of y."""
+        if out is None:
+            out = self._torch.empty_like(x)
+        gleam_dc_forward_aty(x, aty, sens, mask, eta, out, self.dims())
+        return out
 
     def forward_prepared(self, x, y, sens, mask, eta, out=None):
         if out is None:

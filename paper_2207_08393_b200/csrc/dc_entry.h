@@ -14,7 +14,8 @@ enum { RUN_ALL = 0, RUN_PREPARE = 1, RUN_APPLY = 2 };
 // alone (callers that must enqueue something of their own before the step run them first).
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
         const gleam_dims* d, int mode = RUN_ALL, double* dot_rows = nullptr, bool check_only = false,
-        int layout = 0);     // layout: GLEAM_X_CHANNELS | GLEAM_OUT_CHANNELS (two-real-channel image arrays)
+        int layout = 0,      // layout: GLEAM_X_CHANNELS | GLEAM_OUT_CHANNELS (two-real-channel image arrays)
+        const void* aty = nullptr);   // with y == nullptr: out = x - eta (A^H A x - aty), aty = A^H y as an image
 
 // dot_rows (device, one double per image row, B*T*n1): the one-pass 2-D kernel also stores
 // Re<x_row, out_row> of every row it writes, so that a caller's inner product <x, out> needs no

@@ -41,7 +41,17 @@ struct RowArgs {
     // part `plane` further on (plane = T * n0 * n1 * n2).
     int x_planar, out_planar;
     long long plane;
+    // Normal-equations form of the step: when not null (only with z == null), the image A^H y (B,T,n0,n1,n2),
+    // complex interleaved; the kernels that write `out` then store x - eta * (sum - aty).
+    const cf* aty;
 };
+
+// coil sum minus the given A^H y image (element e), if there is one
+__device__ __forceinline__ cf minus_aty(cf acc, const cf* aty, long long e) {
+    if (aty == nullptr) return acc;
+    const cf t = aty[e];
+    return make_float2(acc.x - t.x, acc.y - t.y);
+}
 
 // image-side element e (complex-element offset in the (B,T,V) array) of example b, in either layout
 __device__ __forceinline__ cf load_image(const cf* x, long long e, int planar, int b, long long plane) {
@@ -229,9 +239,11 @@ row_kernel(const RowArgs a) {
                 for (int m = 0; m < R0; ++m) xv[m] = load_image(a.x, x_off + d.j0 + P::BF0 * m, a.x_planar, b0, a.plane);
             }
 #pragma unroll
-            for (int m = 0; m < R0; ++m)
+            for (int m = 0; m < R0; ++m) {
+                const cf av = minus_aty(acc[m], a.aty, x_off + d.j0 + P::BF0 * m);
                 store_image(a.out, x_off + d.j0 + P::BF0 * m,
-                            make_float2(fmaf(-a.eta, acc[m].x, xv[m].x), fmaf(-a.eta, acc[m].y, xv[m].y)), a.out_planar, b0, a.plane);
+                            make_float2(fmaf(-a.eta, av.x, xv[m].x), fmaf(-a.eta, av.y, xv[m].y)), a.out_planar, b0, a.plane);
+            }
         }
     }
 }

@@ -29,6 +29,7 @@ struct TileArgs {
     int C, T, Ts, n0, G, i0_start;
     long long nunits;                         // B*C*T
     int x_planar, out_planar; long long plane; // two-real-channel layout of x / out (see RowArgs)
+    const cf* aty;                            // A^H y image of the normal-equations form, or null (see RowArgs)
 };
 
 template <class PZ, int RY, int BY>
@@ -211,8 +212,10 @@ rowtile_kernel(const TileArgs a) {
     cp_async_wait<0>();
     if (INV && a0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m)
-            store_image(a.out, x_off + jz + PZ::BF0 * m, make_float2(fmaf(-a.eta, acc[m].x, xreg[m].x), fmaf(-a.eta, acc[m].y, xreg[m].y)), a.out_planar, b, a.plane);
+        for (int m = 0; m < R0; ++m) {
+            const cf av = minus_aty(acc[m], a.aty, x_off + jz + PZ::BF0 * m);
+            store_image(a.out, x_off + jz + PZ::BF0 * m, make_float2(fmaf(-a.eta, av.x, xreg[m].x), fmaf(-a.eta, av.y, xreg[m].y)), a.out_planar, b, a.plane);
+        }
     }
 }
 

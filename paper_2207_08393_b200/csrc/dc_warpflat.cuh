@@ -322,7 +322,8 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) {
                 const cf xv = x_at(j + RL * m);
-                const cf ov = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
+                const cf av = minus_aty(acc[m], a.aty, x_off + j + RL * m);
+                const cf ov = make_float2(fmaf(-a.eta, av.x, xv.x), fmaf(-a.eta, av.y, xv.y));
                 store_image(a.out, x_off + j + RL * m, ov, a.out_planar, b, a.plane);
                 if (a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;
             }

@@ -300,7 +300,8 @@ warpline_kernel(const RowArgs a) {
                         const float* xf = reinterpret_cast<const float*>(sX + l * N);
                         xv = (a.x_planar && (N % 4 == 0)) ? make_float2(xf[idx], xf[N + idx]) : sX[l * N + idx];
                     }
-                    const cf ov = make_float2(fmaf(-a.eta, acc[m].x, xv.x), fmaf(-a.eta, acc[m].y, xv.y));
+                    const cf av = minus_aty(acc[m], a.aty, x_off + j + P::BF0 * m);
+                    const cf ov = make_float2(fmaf(-a.eta, av.x, xv.x), fmaf(-a.eta, av.y, xv.y));
                     store_image(a.out, x_off + j + P::BF0 * m, ov, a.out_planar, b, a.plane);
                     if (MODE == ROW_FUSED && a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;
                 }

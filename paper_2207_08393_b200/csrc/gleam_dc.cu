@@ -311,8 +311,9 @@ bool dot_rows_supported(const gleam_dims* d) {
 }
 
 int run(const void* x, const void* y, const void* sens, const float* mask, float eta, void* out,
-        const gleam_dims* d, int mode, double* dot_rows, bool check_only, int layout) {
+        const gleam_dims* d, int mode, double* dot_rows, bool check_only, int layout, const void* aty) {
     if (!d || !mask) return GLEAM_ERR_NULL_POINTER;
+    if (aty && (y || mode != RUN_ALL)) return GLEAM_ERR_BAD_DIMS;      // the given A^H y stands in for y
     if (mode == RUN_PREPARE) {
         if (!y) return GLEAM_ERR_NULL_POINTER;
         x = nullptr; sens = nullptr; out = nullptr;
@@ -333,8 +334,8 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
     const uint64_t sens_b = (uint64_t)L.B * L.C * L.Ts * L.V * sizeof(cf);
     const long long pe = (L.rank == 2) ? L.n2 : (long long)L.n1 * L.n2;
     const uint64_t mask_b = (uint64_t)L.images * (L.separable ? pe : L.V) * sizeof(float);
-    const void* ptrs[6] = {x, y, sens, mask, out, d->workspace};
-    for (int i = 0; i < 6; ++i) {
+    const void* ptrs[7] = {x, y, sens, mask, out, d->workspace, aty};
+    for (int i = 0; i < 7; ++i) {
         if (!ptrs[i]) continue;
         if (((uintptr_t)ptrs[i] & 15) != 0) return GLEAM_ERR_BAD_DIMS;   // 16-byte copies
         rc = check_device_ptr(ptrs[i]);
@@ -347,12 +348,14 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
         if (out == x && ((layout & GLEAM_X_CHANNELS) != 0) != ((layout & GLEAM_OUT_CHANNELS) != 0)) return GLEAM_ERR_ALIAS;
         if (overlaps(out, img_b, sens, sens_b) || overlaps(out, img_b, mask, mask_b)) return GLEAM_ERR_ALIAS;
         if (y && overlaps(out, img_b, y, ksp_b)) return GLEAM_ERR_ALIAS;
+        if (aty && overlaps(out, img_b, aty, img_b)) return GLEAM_ERR_ALIAS;
     }
     if (L.total > 0) {
         const void* w = d->workspace;
         if ((mode != RUN_PREPARE && (overlaps(w, L.total, x, img_b) || overlaps(w, L.total, out, img_b) ||
                                      overlaps(w, L.total, sens, sens_b))) ||
-            overlaps(w, L.total, mask, mask_b) || (y && overlaps(w, L.total, y, ksp_b)))
+            overlaps(w, L.total, mask, mask_b) || (y && overlaps(w, L.total, y, ksp_b)) ||
+            (aty && overlaps(w, L.total, aty, img_b)))
             return GLEAM_ERR_ALIAS;
     }
     if (check_only) return GLEAM_OK;          // every argument check has passed; nothing is enqueued
@@ -368,6 +371,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
     ra.C = L.C; ra.T = L.T; ra.Ts = L.Ts; ra.RPB = L.n0 * L.n1;
     ra.x_planar = (layout & GLEAM_X_CHANNELS) ? 1 : 0; ra.out_planar = (layout & GLEAM_OUT_CHANNELS) ? 1 : 0;
     ra.plane = (long long)L.T * L.V;
+    ra.aty = (const cf*)aty;
     ColArgs ca{};
     ca.C = L.C; ca.T = L.T; ca.rank = L.rank; ca.n0 = L.n0; ca.n1 = L.n1; ca.n2 = L.n2;
 
@@ -415,7 +419,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
             ra.dot_rows = dot_rows;
             LAUNCH(GLEAM_K_ROW_FUSED, op2->row(ROW_FUSED, ra, s));
         } else {
-            if (L.fused && !y && layout == 0) {
+            if (L.fused && !y && !aty && layout == 0) {
                 // one persistent kernel walks all slabs; its counters start from zero
                 FusedArgs fa{};
                 fa.x = (const cf*)x; fa.sens = (const cf*)sens; fa.out = (cf*)out; fa.W = (cf*)(ws + L.off_ring);
@@ -439,7 +443,7 @@ int run(const void* x, const void* y, const void* sens, const float* mask, float
                     ta.x = (const cf*)x; ta.sens = (const cf*)sens; ta.out = (cf*)out; ta.V = W; ta.mask = mask;
                     ta.zin = z; ta.zidx = ca.zidx; ta.m2c = ca.m2c; ta.zstart = ca.zstart; ta.eta = eta; ta.scale2 = 1.0f / (float)pe;
                     ta.C = L.C; ta.T = L.T; ta.Ts = L.Ts; ta.n0 = L.n0; ta.G = g; ta.i0_start = i0; ta.nunits = L.units;
-                    ta.x_planar = ra.x_planar; ta.out_planar = ra.out_planar; ta.plane = ra.plane;
+                    ta.x_planar = ra.x_planar; ta.out_planar = ra.out_planar; ta.plane = ra.plane; ta.aty = ra.aty;
                     LAUNCH(GLEAM_K_ROW_FWD, pair->fwd(ta, L.images, s));
                     LAUNCH(GLEAM_K_COL_MID_SEP, pair->mid(ta, s));
                     LAUNCH(GLEAM_K_ROW_INV, pair->inv(ta, L.images, s));
@@ -620,6 +624,12 @@ GLEAM_API int gleam_dc_adjoint(const void* y, const void* sens, const float* mas
     const uint64_t img_b = (uint64_t)dims->batch * dims->frames * dims->n[0] * dims->n[1] * dims->n[2] * sizeof(gleam::cf);
     if (cudaMemsetAsync(out, 0, img_b, (cudaStream_t)dims->stream) != cudaSuccess) return GLEAM_ERR_CUDA;
     return gleam::run(out, y, sens, mask, 1.0f, out, dims);     // 0 - 1 * A^H (A 0 - y), in place
+}
+
+GLEAM_API int gleam_dc_forward_aty(const void* x, const void* aty, const void* sens, const float* mask, float eta,
+                                   void* out, const gleam_dims* dims) {
+    if (!aty) return GLEAM_ERR_NULL_POINTER;
+    return gleam::run(x, nullptr, sens, mask, eta, out, dims, gleam::RUN_ALL, nullptr, false, 0, aty);
 }
 
 GLEAM_API int gleam_dc_prepare(const void* y, const float* mask, const gleam_dims* dims) {

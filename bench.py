@@ -429,6 +429,46 @@ def run_ours(args, w):
                     "value": w.voxel_coils * chain / (step_ms * 1e-3), "unit": UNIT,
                     "what": "1 gleam_dc_prepare + %d gleam_dc_forward_prepared per step, VJP chain as in the main number" % chain}
 
+    # ---- the same chain in normal-equations form: A^H y once per step, then steps that cost a VJP call ----
+    aty_chain = None
+    if True:
+        aty_buf = torch.empty_like(tx)
+
+        def forward_chain_aty():
+            dc.adjoint(ty, ts, tm, aty_buf)
+            src = tx
+            for i in range(chain):
+                dst = out if i % 2 == 0 else out2
+                dc.forward_aty(src, aty_buf, ts, tm, w.eta, dst)
+                src = dst
+
+        forward_chain(); torch.cuda.synchronize()
+        ref_last = (out if (chain - 1) % 2 == 0 else out2).clone()
+        forward_chain_aty(); torch.cuda.synchronize()
+        got_last = out if (chain - 1) % 2 == 0 else out2
+        dev_rel = float((got_last - ref_last).abs().pow(2).sum().sqrt() / ref_last.abs().pow(2).sum().sqrt())
+        assert dev_rel < 2e-5 * chain, "normal-equations chain differs from the plain chain: %g" % dev_rel
+        af, ad = 0.0, 0.0
+        for _ in range(prof_steps):
+            if flush is not None:
+                flush.fill_(1)
+            ef[0].record(stream); dc.adjoint(ty, ts, tm, aty_buf)
+            ef[1].record(stream)
+            src = tx
+            for i in range(chain):
+                dst = out if i % 2 == 0 else out2
+                dc.forward_aty(src, aty_buf, ts, tm, w.eta, dst)
+                src = dst
+            ef[2].record(stream); torch.cuda.synchronize()
+            ad += ef[0].elapsed_time(ef[1]) / prof_steps
+            af += ef[1].elapsed_time(ef[2]) / prof_steps
+        step_ms = ad + af + split[1] * chain
+        aty_chain = {"adjoint_us": ad * 1e3, "forward_us_per_call": af / chain * 1e3, "ms_per_step": step_ms,
+                     "value": w.voxel_coils * chain / (step_ms * 1e-3), "unit": UNIT,
+                     "rel_l2_against_plain_chain": dev_rel,
+                     "what": "1 gleam_dc_adjoint (A^H y) + %d gleam_dc_forward_aty per step, VJP chain as in the main number" % chain}
+        del aty_buf
+
     # ---- the same steps without the L2 flush (problems that fit in L2: both figures are reported) ----
     warm = None
     if flush is not None:
@@ -500,6 +540,15 @@ def run_ours(args, w):
                     "measured_us": ms * 1e3, "frac": max(t_b, t_f) / (ms * 1e-3),
                     "frac_with_measured_fp32_peak": max(t_b, flops / (alu_measured * 1e12)) / (ms * 1e-3)}
 
+    if aty_chain is not None:       # x, A^H y, S, mask in; out: no measurements are read
+        nbytes, flops = call_roofline(w, False)
+        nbytes += w.batch * w.frames * w.V * 8
+        t_b, t_f = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (alu_peak * 1e12)
+        ms = aty_chain["forward_us_per_call"] * 1e-3
+        ns["forward_aty"] = {"min_bytes": nbytes, "fft_flops": flops, "hbm_us": t_b * 1e6, "fp32_us": t_f * 1e6,
+                             "measured_us": ms * 1e3, "frac": max(t_b, t_f) / (ms * 1e-3),
+                             "frac_with_measured_fp32_peak": max(t_b, flops / (alu_measured * 1e12)) / (ms * 1e-3)}
+
     # ---- CPU baseline: the oracle, once, on the host cores of the machine ---------------------------
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -540,6 +589,7 @@ def run_ours(args, w):
         "fp32_peak": {"derived_tflops": alu_peak, "measured_tflops": alu_measured,
                       "how": "derived: 148 SMs x 128 lanes x 2 flop x sm_max_mhz; measured: independent FMA chains, no memory traffic"},
         "prepared_chain": prepared,
+        "normal_equations_chain": aty_chain,
         "warm_l2": warm,
         "two_channel_layout": layout_cost,
         "kernels": kernels,

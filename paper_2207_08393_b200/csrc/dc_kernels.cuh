@@ -46,11 +46,13 @@ struct RowArgs {
     const cf* aty;
 };
 
-// coil sum minus the given A^H y image (element e), if there is one
-__device__ __forceinline__ cf minus_aty(cf acc, const cf* aty, long long e) {
-    if (aty == nullptr) return acc;
+// Start value of the coil sum of image element e: minus the given A^H y, if there is one.  Taking it as the
+// start value puts its load at the beginning of the coil loop, where its latency costs nothing, and needs no
+// register of its own.
+__device__ __forceinline__ cf coil_sum_start(const cf* aty, long long e) {
+    if (aty == nullptr) return make_float2(0.f, 0.f);
     const cf t = aty[e];
-    return make_float2(acc.x - t.x, acc.y - t.y);
+    return make_float2(-t.x, -t.y);
 }
 
 // image-side element e (complex-element offset in the (B,T,V) array) of example b, in either layout
@@ -122,7 +124,7 @@ row_kernel(const RowArgs a) {
     cf xv[R0], acc[R0];
     if (MODE != ROW_FWD) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
+        for (int m = 0; m < R0; ++m) acc[m] = act0 ? coil_sum_start(a.aty, x_off + d.j0 + P::BF0 * m) : make_float2(0.f, 0.f);
     }
     if (MODE != ROW_INV) {
         if (act0) {
@@ -240,7 +242,7 @@ row_kernel(const RowArgs a) {
             }
 #pragma unroll
             for (int m = 0; m < R0; ++m) {
-                const cf av = minus_aty(acc[m], a.aty, x_off + d.j0 + P::BF0 * m);
+                const cf av = acc[m];
                 store_image(a.out, x_off + d.j0 + P::BF0 * m,
                             make_float2(fmaf(-a.eta, av.x, xv[m].x), fmaf(-a.eta, av.y, xv[m].y)), a.out_planar, b0, a.plane);
             }

@@ -107,7 +107,7 @@ rowtile_kernel(const TileArgs a) {
     cf xreg[R0], acc[R0];
     if (a0) {
 #pragma unroll
-        for (int m = 0; m < R0; ++m) { xreg[m] = load_image(a.x, x_off + jz + PZ::BF0 * m, a.x_planar, b, a.plane); acc[m] = make_float2(0.f, 0.f); }
+        for (int m = 0; m < R0; ++m) { xreg[m] = load_image(a.x, x_off + jz + PZ::BF0 * m, a.x_planar, b, a.plane); acc[m] = INV ? coil_sum_start(a.aty, x_off + jz + PZ::BF0 * m) : make_float2(0.f, 0.f); }
     }
     issue_s(0);
     // pass 3: the column values of the first coil (one kz column per thread; THREADS >= NZ is not
@@ -213,7 +213,7 @@ rowtile_kernel(const TileArgs a) {
     if (INV && a0) {
 #pragma unroll
         for (int m = 0; m < R0; ++m) {
-            const cf av = minus_aty(acc[m], a.aty, x_off + jz + PZ::BF0 * m);
+            const cf av = acc[m];
             store_image(a.out, x_off + jz + PZ::BF0 * m, make_float2(fmaf(-a.eta, av.x, xreg[m].x), fmaf(-a.eta, av.y, xreg[m].y)), a.out_planar, b, a.plane);
         }
     }

@@ -192,7 +192,7 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 
         cf acc[R0];
 #pragma unroll
-        for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
+        for (int m = 0; m < R0; ++m) acc[m] = (row_ok && q == 0) ? coil_sum_start(a.aty, x_off + j + RL * m) : make_float2(0.f, 0.f);
         cf sf[R0];                       // sensitivities of the next forward image-side stage
         if (nc > 0) load_sens(sf, 0);
 #ifdef GLEAM_TRACE
@@ -322,7 +322,7 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 #pragma unroll
             for (int m = 0; m < R0; ++m) {
                 const cf xv = x_at(j + RL * m);
-                const cf av = minus_aty(acc[m], a.aty, x_off + j + RL * m);
+                const cf av = acc[m];
                 const cf ov = make_float2(fmaf(-a.eta, av.x, xv.x), fmaf(-a.eta, av.y, xv.y));
                 store_image(a.out, x_off + j + RL * m, ov, a.out_planar, b, a.plane);
                 if (a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;

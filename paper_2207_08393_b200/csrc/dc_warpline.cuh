@@ -174,7 +174,8 @@ warpline_kernel(const RowArgs a) {
             for (int m = 0; m < R0; ++m) xreg[m] = load_image(a.x, x_off + j + P::BF0 * m, a.x_planar, b, a.plane);
         }
 #pragma unroll
-        for (int m = 0; m < R0; ++m) acc[m] = make_float2(0.f, 0.f);
+        for (int m = 0; m < R0; ++m)
+            acc[m] = (MODE != ROW_FWD && a0 && row_ok) ? coil_sum_start(a.aty, x_off + j + P::BF0 * m) : make_float2(0.f, 0.f);
 
         for (int c = 0; c < a.C; ++c) {
             const int buf = c & 1;
@@ -300,7 +301,7 @@ warpline_kernel(const RowArgs a) {
                         const float* xf = reinterpret_cast<const float*>(sX + l * N);
                         xv = (a.x_planar && (N % 4 == 0)) ? make_float2(xf[idx], xf[N + idx]) : sX[l * N + idx];
                     }
-                    const cf av = minus_aty(acc[m], a.aty, x_off + j + P::BF0 * m);
+                    const cf av = acc[m];
                     const cf ov = make_float2(fmaf(-a.eta, av.x, xv.x), fmaf(-a.eta, av.y, xv.y));
                     store_image(a.out, x_off + j + P::BF0 * m, ov, a.out_planar, b, a.plane);
                     if (MODE == ROW_FUSED && a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;

@@ -314,6 +314,40 @@ def run_ours(args, w):
         step()
     barrier()
 
+    # ---- the launches of a step, captured once as a CUDA graph and replayed (the calls are a few tens of
+    # microseconds each, so enqueueing them one by one from Python would be part of the measurement) ----
+    use_graph = args.launch == "graph" and not args.kernels_only
+    graph_pool = []
+
+    def replayed(fn):
+        """fn's launches as a CUDA graph on the current stream; fn itself when graphs are off or the capture fails."""
+        if not use_graph:
+            return fn, None
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                fn()                                   # first use on this stream outside the capture
+                torch.cuda.synchronize()
+                n0 = g.gleam_dc_launch_count()
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=side):
+                    fn()
+                n1 = g.gleam_dc_launch_count()
+            stream.wait_stream(side)
+            torch.cuda.synchronize()
+            graph_pool.append(gr)
+            return gr.replay, int(n1 - n0)
+        except Exception as e:                         # noqa: BLE001
+            sys.stderr.write("graph capture failed (%s): launching eagerly\n" % e)
+            return fn, None
+
+    step_eager = step
+    step, step_launches = replayed(step_eager)
+    for _ in range(3):
+        step()
+    barrier()
+
     # ---- device-resident timed region -------------------------------------------------------
     launches0 = g.gleam_dc_launch_count()
     t_begin = time.time()
@@ -337,7 +371,7 @@ def run_ours(args, w):
             b.record(stream)
         barrier()
         local_ms = sum(a.elapsed_time(b) for a, b in evs)
-    launches = g.gleam_dc_launch_count() - launches0
+    launches = g.gleam_dc_launch_count() - launches0 if step_launches is None else step_launches * args.steps
     t_end = time.time()
     total_ms, total_units = aggregate(local_ms, w.voxel_coils * chain * args.steps, world, dist, dev)
     value = total_units / (total_ms * 1e-3)
@@ -358,7 +392,7 @@ def run_ours(args, w):
     for _ in range(prof_steps):
         if flush is not None:
             flush.fill_(1)
-        step()
+        step_eager()
     prof = g.gleam_dc_profile_end()
     kernels = {}
     for cls, (ms, cnt) in prof.items():
@@ -371,11 +405,13 @@ def run_ours(args, w):
     # forward / vjp split (events around whole calls)
     ef = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
     split = [0.0, 0.0]
+    forward_chain_r, _ = replayed(forward_chain)
+    vjp_chain_r, _ = replayed(vjp_chain)
     for _ in range(prof_steps):
         if flush is not None:
             flush.fill_(1)
-        ef[0].record(stream); forward_chain()
-        ef[1].record(stream); vjp_chain()
+        ef[0].record(stream); forward_chain_r()
+        ef[1].record(stream); vjp_chain_r()
         ef[2].record(stream); torch.cuda.synchronize()
         split[0] += ef[0].elapsed_time(ef[1]) / prof_steps / chain      # per call
         split[1] += ef[1].elapsed_time(ef[2]) / prof_steps / chain
@@ -393,7 +429,7 @@ def run_ours(args, w):
 
     lay = [0.0, 0.0]
     for _ in range(prof_steps):
-        for k, fn in enumerate((vjp_chain, vjp_chain_channels)):
+        for k, fn in enumerate((vjp_chain_r, replayed(vjp_chain_channels)[0])):
             if flush is not None:
                 flush.fill_(1)
             ef[0].record(stream); fn()
@@ -418,10 +454,11 @@ def run_ours(args, w):
         forward_chain_prepared(); torch.cuda.synchronize()
         assert torch.equal(ref_last, out if (chain - 1) % 2 == 0 else out2), "prepared chain differs"
         pf = 0.0
+        forward_chain_prepared_r, _ = replayed(forward_chain_prepared)
         for _ in range(prof_steps):
             if flush is not None:
                 flush.fill_(1)
-            ef[0].record(stream); forward_chain_prepared()
+            ef[0].record(stream); forward_chain_prepared_r()
             ef[1].record(stream); torch.cuda.synchronize()
             pf += ef[0].elapsed_time(ef[1]) / prof_steps
         step_ms = pf + split[1] * chain
@@ -449,16 +486,21 @@ def run_ours(args, w):
         dev_rel = float((got_last - ref_last).abs().pow(2).sum().sqrt() / ref_last.abs().pow(2).sum().sqrt())
         assert dev_rel < 2e-5 * chain, "normal-equations chain differs from the plain chain: %g" % dev_rel
         af, ad = 0.0, 0.0
-        for _ in range(prof_steps):
-            if flush is not None:
-                flush.fill_(1)
-            ef[0].record(stream); dc.adjoint(ty, ts, tm, aty_buf)
-            ef[1].record(stream)
+
+        def aty_steps():
             src = tx
             for i in range(chain):
                 dst = out if i % 2 == 0 else out2
                 dc.forward_aty(src, aty_buf, ts, tm, w.eta, dst)
                 src = dst
+
+        adjoint_r, _ = replayed(lambda: dc.adjoint(ty, ts, tm, aty_buf))
+        aty_steps_r, _ = replayed(aty_steps)
+        for _ in range(prof_steps):
+            if flush is not None:
+                flush.fill_(1)
+            ef[0].record(stream); adjoint_r()
+            ef[1].record(stream); aty_steps_r()
             ef[2].record(stream); torch.cuda.synchronize()
             ad += ef[0].elapsed_time(ef[1]) / prof_steps
             af += ef[1].elapsed_time(ef[2]) / prof_steps
@@ -576,6 +618,7 @@ def run_ours(args, w):
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "description": w.description, "step": "%d chained gleam_dc_forward + %d chained gleam_dc_vjp" % (chain, chain),
+                   "launch": "one CUDA graph per step, captured from the same C-ABI calls and replayed" if step_launches is not None else "eager, call by call",
                    "voxel_coils_per_step": w.voxel_coils * chain, "e2e_step": "1 forward + 1 vjp with host buffers", "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "l2": "inputs exceed L2" if flush is None else "256 MB L2 flush before every step (chain)",
                    "mask": "general (B,T,n0,n1,n2) array" if full_mask else "readout-invariant"},
@@ -818,6 +861,8 @@ def main():
     ap.add_argument("--kernels-only", action="store_true",
                     help="profiler run: warm-up and timed steps only, then a short JSON line (no per-kernel pass, no "
                          "end-to-end leg, no CPU baseline)")
+    ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
+                    help="graph: the step's launches are captured once and replayed; eager: enqueued call by call")
     ap.add_argument("--calls", default="both", choices=["both", "forward", "vjp"], help="which calls a step makes")
     ap.add_argument("--print-sources-digest", action="store_true", help="print the digest that keys profiles/dram_traffic.json")
     ap.add_argument("--method", default="dc", choices=["dc", "modl"],

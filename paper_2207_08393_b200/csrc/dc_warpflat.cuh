@@ -64,7 +64,7 @@ struct WarpFlat {
 // One block per SM also keeps a dependent launch from moving in next to the running one warp by warp, which
 // would fill the schedulers unevenly.
 template <class P, bool HAS_Z, bool SMW>
-__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : 16)
+__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : (P::RL == 32 ? 12 : 13))
 warpflat_kernel(const RowArgs a, const int nwhole) {
     grid_dependency_wait();
     grid_launch_dependents();

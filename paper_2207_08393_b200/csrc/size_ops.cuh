@@ -116,7 +116,7 @@ inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
     // SM: the groups beyond 4 k are split by coils over four warps each, one per scheduler.  (Measured on cine-shaped
     // problems, per call: 13 groups per SM 18.7 -> 16.6 us, 12 per SM 18.7 -> 15.3 us; up to 7 per SM single-warp
     // blocks are faster, 11.3 against 12.7 us.)
-    {
+    if constexpr (P::RL <= 16) {        // 32-point butterflies need more registers than 16 warps per SM leave
         using WS = WarpFlat<P, HAS_Z, true>;
         static PerDevice attrs_done;
         int sms = 0, dev = 0;
@@ -146,11 +146,23 @@ inline bool flat_enabled() {
     return v == 1;
 }
 
+// Stage plan of the one-pass kernel with units numbered across coils, per length: the last radix RL (8, 16 or
+// 32 = butterflies of the first stage per line) where that kernel is used, 0 where the plain plan stays.
+template <int N> struct FlatRL { static constexpr int value = 0; };
+template <> struct FlatRL<160> { static constexpr int value = 16; };    // 10 x 16
+template <> struct FlatRL<320> { static constexpr int value = 32; };    // 10 x 32
+template <class P> struct FlatPlan {
+    static constexpr int RL = FlatRL<P::N>::value;
+    using type = Plan<P::N, RL ? P::N / RL : P::R0, RL ? RL : P::R1, RL ? 1 : P::R2>;
+};
+
 template <class P, int MODE>
 inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
-    if constexpr (MODE == ROW_FUSED && WarpFlat<P, false>::ELIGIBLE) {
+    if constexpr (MODE == ROW_FUSED && FlatRL<P::N>::value != 0) {
+        using PF = typename FlatPlan<P>::type;
+        static_assert(WarpFlat<PF, false>::ELIGIBLE, "not a plan the coil-numbered kernel takes");
         // the numbering across coils pays once a round of 32 units spans more than one coil
-        if (flat_enabled() && a.C >= 2) return a.z != nullptr ? launch_warpflat_z<P, true>(a, s) : launch_warpflat_z<P, false>(a, s);
+        if (flat_enabled() && a.C >= 2) return a.z != nullptr ? launch_warpflat_z<PF, true>(a, s) : launch_warpflat_z<PF, false>(a, s);
     }
     if (MODE == ROW_FUSED && a.z != nullptr) return launch_warpline_z<P, MODE, true>(a, s);
     return launch_warpline_z<P, MODE, false>(a, s);

@@ -19,10 +19,6 @@
 
 namespace gleam {
 
-#ifdef GLEAM_TRACE
-__device__ long long g_trace[8 * 8192];
-__device__ __forceinline__ long long trace_now() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#endif
 
 template <class P, bool HAS_Z, bool SMW = false>
 struct WarpFlat {
@@ -63,15 +59,14 @@ struct WarpFlat {
 // coil sums are added in warp order through shared memory.  A quarter of the extra work lands on every scheduler.
 // One block per SM also keeps a dependent launch from moving in next to the running one warp by warp, which
 // would fill the schedulers unevenly.
-template <class P, bool HAS_Z, bool SMW>
-__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : (P::RL == 32 ? 12 : 13))
+// HAS_ATY: the coil sum starts from minus the given A^H y image (normal-equations form of the step; never together
+// with z).  A template parameter, not a run-time test of a.aty: with the test in the code the plain call measured
+// 11 % slower (17.7 against 16.0 us), although it never takes that branch.
+template <class P, bool HAS_Z, bool SMW, bool HAS_ATY>
+__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : (P::RL == 32 ? 12 : 16))
 warpflat_kernel(const RowArgs a, const int nwhole) {
     grid_dependency_wait();
     grid_launch_dependents();
-#ifdef GLEAM_TRACE
-    const long long tr_t0 = trace_now();
-    long long tr_t1 = 0;
-#endif
     using WF = WarpFlat<P, HAS_Z, SMW>;
     constexpr int N = P::N, R0 = P::R0, RL = P::RL, LW = WF::LW, UPC = WF::UPC, US = WF::USTRIDE, SLOTS = WF::SLOTS;
     constexpr int KCAP = WF::KCAP, KSTRIDE = WF::KSTRIDE, KTILE = WF::KTILE, ZS = WF::ZS, MS = WF::MS;
@@ -192,12 +187,9 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 
         cf acc[R0];
 #pragma unroll
-        for (int m = 0; m < R0; ++m) acc[m] = (row_ok && q == 0) ? coil_sum_start(a.aty, x_off + j + RL * m) : make_float2(0.f, 0.f);
+        for (int m = 0; m < R0; ++m) acc[m] = (HAS_ATY && row_ok && q == 0) ? coil_sum_start(a.aty, x_off + j + RL * m) : make_float2(0.f, 0.f);
         cf sf[R0];                       // sensitivities of the next forward image-side stage
         if (nc > 0) load_sens(sf, 0);
-#ifdef GLEAM_TRACE
-        tr_t1 = trace_now();
-#endif
         int af = 0, ai = 0;              // next coil of the forward / of the inverse image-side stage
 
         for (int br = 0; br < rounds; ++br) {
@@ -333,14 +325,6 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
             if (j == 0 && row_ok) a.dot_rows[row] = dsum;
         }
     }
-#ifdef GLEAM_TRACE
-    if ((threadIdx.x & 31) == 0) {
-        unsigned sm_, w_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); asm volatile("mov.u32 %0, %%warpid;" : "=r"(w_));
-        const int slot = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) & 8191;
-        g_trace[8 * slot + 0] = tr_t0; g_trace[8 * slot + 1] = tr_t1; g_trace[8 * slot + 2] = trace_now();
-        g_trace[8 * slot + 3] = sm_; g_trace[8 * slot + 4] = w_; g_trace[8 * slot + 5] = blockIdx.x; g_trace[8 * slot + 6] = threadIdx.x >> 5;
-    }
-#endif
 }
 
 }  // namespace gleam

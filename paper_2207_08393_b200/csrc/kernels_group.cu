@@ -8,9 +8,3 @@ namespace gleam {
 #include "sizes.def"
 #undef GLEAM_SIZE
 }  // namespace gleam
-
-#if defined(GLEAM_TRACE) && GLEAM_GROUP == 2
-extern "C" __attribute__((visibility("default"))) int gleam_trace_read(long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, gleam::g_trace, sizeof(long long) * n);
-}
-#endif

@@ -101,15 +101,15 @@ inline bool split_enabled() {
 }
 
 // the one-pass kernel with the k-space units numbered across the coils (dc_warpflat.cuh)
-template <class P, bool HAS_Z>
-inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
+template <class P, bool HAS_Z, bool HAS_ATY>
+inline cudaError_t launch_warpflat_zy(const RowArgs& a, cudaStream_t s) {
     using WF = WarpFlat<P, HAS_Z, false>;
     static PerDevice attr_done;
     static PerDevice slots_cache;
-    cudaError_t e = ensure_smem(warpflat_kernel<P, HAS_Z, false>, WF::WARP_BYTES, attr_done);
+    cudaError_t e = ensure_smem(warpflat_kernel<P, HAS_Z, false, HAS_ATY>, WF::WARP_BYTES, attr_done);
     if (e != cudaSuccess) return e;
     int slots = 0;
-    if ((e = resident_slots(warpflat_kernel<P, HAS_Z, false>, 32, WF::WARP_BYTES, slots_cache, &slots)) != cudaSuccess) return e;
+    if ((e = resident_slots(warpflat_kernel<P, HAS_Z, false, HAS_ATY>, 32, WF::WARP_BYTES, slots_cache, &slots)) != cudaSuccess) return e;
     const long long groups = (a.nrows + WF::LW - 1) / WF::LW;
     if (groups <= 0) return cudaSuccess;
     // One round of 8 to 16 groups per SM: one block per SM that holds all its warps.  4 k + 1 (or 4 k + 2) groups per
@@ -130,14 +130,19 @@ inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
             // with z the split groups were measured slower than single-warp blocks (13 groups per SM: 25.2 against
             // 24.7 us per call), whole groups alone faster (12 per SM: 22.5 against 24.5 us)
             if (warps <= 16 && bytes <= 227 * 1024 && !(HAS_Z && nsplit > 0)) {
-                if ((e = ensure_smem(warpflat_kernel<P, HAS_Z, true>, 16 * WS::WARP_BYTES, attrs_done)) != cudaSuccess) return e;
-                return launch_overlapped(true, warpflat_kernel<P, HAS_Z, true>, dim3((unsigned)sms), dim3(32 * warps), bytes, s, a, nwhole);
+                if ((e = ensure_smem(warpflat_kernel<P, HAS_Z, true, HAS_ATY>, 16 * WS::WARP_BYTES, attrs_done)) != cudaSuccess) return e;
+                return launch_overlapped(true, warpflat_kernel<P, HAS_Z, true, HAS_ATY>, dim3((unsigned)sms), dim3(32 * warps), bytes, s, a, nwhole);
             }
         }
     }
     long long blocks = groups;
     if (blocks > slots) blocks = slots;
-    return launch_overlapped(groups <= slots, warpflat_kernel<P, HAS_Z, false>, dim3((unsigned)blocks), dim3(32), WF::WARP_BYTES, s, a, 1);
+    return launch_overlapped(groups <= slots, warpflat_kernel<P, HAS_Z, false, HAS_ATY>, dim3((unsigned)blocks), dim3(32), WF::WARP_BYTES, s, a, 1);
+}
+template <class P, bool HAS_Z>
+inline cudaError_t launch_warpflat_z(const RowArgs& a, cudaStream_t s) {
+    if constexpr (!HAS_Z) { if (a.aty != nullptr) return launch_warpflat_zy<P, false, true>(a, s); }
+    return launch_warpflat_zy<P, HAS_Z, false>(a, s);
 }
 // GLEAM_NO_FLAT=1 keeps the plain warp-resident kernel for those lengths (tuning aid, read once).
 inline bool flat_enabled() {

@@ -130,7 +130,9 @@ inline cudaError_t launch_warpflat_zy(const RowArgs& a, cudaStream_t s) {
             // with z the split groups were measured slower than single-warp blocks (13 groups per SM: 25.2 against
             // 24.7 us per call), whole groups alone faster (12 per SM: 22.5 against 24.5 us)
             if (warps <= 16 && bytes <= 227 * 1024 && !(HAS_Z && nsplit > 0)) {
-                if ((e = ensure_smem(warpflat_kernel<P, HAS_Z, true, HAS_ATY>, 16 * WS::WARP_BYTES, attrs_done)) != cudaSuccess) return e;
+                // the attribute is set once, to what the largest block of this kernel can ask for
+                constexpr size_t SMEM_CAP = 227 * 1024;
+                if ((e = ensure_smem(warpflat_kernel<P, HAS_Z, true, HAS_ATY>, 16 * WS::WARP_BYTES < SMEM_CAP ? 16 * WS::WARP_BYTES : SMEM_CAP, attrs_done)) != cudaSuccess) return e;
                 return launch_overlapped(true, warpflat_kernel<P, HAS_Z, true, HAS_ATY>, dim3((unsigned)sms), dim3(32 * warps), bytes, s, a, nwhole);
             }
         }
@@ -153,9 +155,20 @@ inline bool flat_enabled() {
 
 // Stage plan of the one-pass kernel with units numbered across coils, per length: the last radix RL (8, 16 or
 // 32 = butterflies of the first stage per line) where that kernel is used, 0 where the plain plan stays.
+// Measured per call against the plain warp-resident kernel (VJP, 4 x 8 coils x 256 rows / 8 x 16 coils x 512 rows):
+// 80: 6.8 / 17.4 against 8.6 / 29.3 us; 96: 6.3 / 19.2 against 9.2 / 32.9; 128: 7.4 / 24.7 against 10.2 / 40.3;
+// 48: equal for the VJP, forward 24.7 against 33.5; 160 and 320: the cine and brain workloads.
 template <int N> struct FlatRL { static constexpr int value = 0; };
 template <> struct FlatRL<160> { static constexpr int value = 16; };    // 10 x 16
 template <> struct FlatRL<320> { static constexpr int value = 32; };    // 10 x 32
+template <> struct FlatRL<128> { static constexpr int value = 16; };    // 8 x 16
+template <> struct FlatRL<192> { static constexpr int value = 32; };    // 6 x 32
+template <> struct FlatRL<96> { static constexpr int value = 16; };     // 6 x 16
+template <> struct FlatRL<80> { static constexpr int value = 16; };     // 5 x 16
+template <> struct FlatRL<48> { static constexpr int value = 8; };      // 6 x 8
+// lengths whose plain plan already keeps most lanes busy: the coil-numbered kernel only where it measured faster,
+// the call with z (192: forward 25 against 50 us, VJP 50 against 46 us on 8 x 16 coils x 512 rows)
+template <int N> struct FlatOnlyWithZ { static constexpr bool value = (N == 192); };
 template <class P> struct FlatPlan {
     static constexpr int RL = FlatRL<P::N>::value;
     using type = Plan<P::N, RL ? P::N / RL : P::R0, RL ? RL : P::R1, RL ? 1 : P::R2>;
@@ -167,7 +180,8 @@ inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
         using PF = typename FlatPlan<P>::type;
         static_assert(WarpFlat<PF, false>::ELIGIBLE, "not a plan the coil-numbered kernel takes");
         // the numbering across coils pays once a round of 32 units spans more than one coil
-        if (flat_enabled() && a.C >= 2) return a.z != nullptr ? launch_warpflat_z<PF, true>(a, s) : launch_warpflat_z<PF, false>(a, s);
+        if (flat_enabled() && a.C >= 2 && (a.z != nullptr || !FlatOnlyWithZ<P::N>::value))
+            return a.z != nullptr ? launch_warpflat_z<PF, true>(a, s) : launch_warpflat_z<PF, false>(a, s);
     }
     if (MODE == ROW_FUSED && a.z != nullptr) return launch_warpline_z<P, MODE, true>(a, s);
     return launch_warpline_z<P, MODE, false>(a, s);

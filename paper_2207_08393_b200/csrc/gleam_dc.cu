@@ -157,10 +157,11 @@ struct Layout {
     int R, L2, L3;
 };
 
-// Ring size and lags of the fused kernel, in slabs.  The groups of an SM take about four steps per
-// item and one block per SM is resident, so about three periods of items are in flight: P2 follows
-// P1 by L2 = 2 periods, P3 by L3 = 4, and the ring holds R = 8 slabs (42 MB for 8 coils of 320 x 256,
-// inside the 126 MB L2).  GLEAM_FUSED_RING="R,L2,L3" overrides (tuning aid, read once).
+// Ring size and lags of the fused kernel, in slabs: P2 follows P1 by L2 = 2 periods, P3 by L3 = 4, and the ring
+// holds R = 8 slabs (42 MB for 8 coils of 320 x 256).  Larger settings were measured faster per VJP call on the
+// 320 x 320 x 256 volume ((8, 2, 4) 2.36 ms, (12, 3, 6) 2.04 ms, (16, 4, 8) 1.81 ms), but with (16, 4, 8) repeated
+// calls on a 16-slab problem did not give identical bits (cause not found), so the setting whose tests pass stays the
+// default.  GLEAM_FUSED_RING="R,L2,L3" overrides (timing aid, read once).
 static void fused_ring(int* R, int* L2, int* L3) {
     static int v[3] = {0, 0, 0};
     if (v[0] == 0) {
@@ -171,8 +172,8 @@ static void fused_ring(int* R, int* L2, int* L3) {
     }
     *R = v[0]; *L2 = v[1]; *L3 = v[2];
 }
-// The persistent kernel is opt-in: measured on knee3d it is slower than the three whole-volume passes
-// (1.90 ms against 1.77 ms per VJP call), so the default keeps those.  GLEAM_FUSED=1 in the environment
+// The persistent kernel is opt-in: measured on the 320 x 320 x 256 volume it is slower than the three whole-volume
+// passes (2.36 ms against 1.77-1.85 ms per VJP call at the default ring), so the default keeps those.  GLEAM_FUSED=1 in the environment
 // or gleam_dc_set_fused(1) selects it; the choice changes the workspace layout, so it is made before
 // gleam_dc_workspace_size.
 static std::atomic<int> g_fused_on{-1};

@@ -23,7 +23,7 @@ def fused_on():
 
 @pytest.mark.parametrize("B,C,T,n", [
     (1, 2, 1, (4, 64, 256)),        # fewer slabs than ring slots
-    (1, 3, 1, (20, 64, 256)),       # odd coil count (groups of 2 and 1 coils), several ring turns
+    (1, 3, 1, (40, 64, 256)),       # odd coil count (groups of 2 and 1 coils), several ring turns
     (2, 1, 2, (6, 128, 256)),       # one coil: the second compute group only joins the coil sum; batch and frames
     (1, 8, 1, (12, 320, 256)),      # the knee3d phase-encode plane
 ])

@@ -392,3 +392,18 @@ def test_adjoint_is_the_zero_filled_image(oracle, case):
     got = got.astype(np.complex128)
     rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
     assert rel <= 2e-5 and np.abs(got - ref).max() <= 1e-4 * np.abs(ref).max(), rel
+
+
+# ----------------------------------------------------------------------------------------------
+# single-round launches of the one-pass kernel with numbered k-space units: one block per SM, with and
+# without groups split by coils over four warps
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("C,T,R", [
+    (8, 18, 192),      # 12 groups per SM on 148 SMs: whole groups only, also for the call with z
+    (6, 14, 192),      # 10 groups per SM: two groups per SM split over four warps each; coils not a multiple of four
+    (5, 20, 192),      # 13 groups per SM: one split group, quarters of 1, 1, 1 and 2 coils
+    (4, 12, 160),      # 7 groups per SM: single-warp blocks
+])
+def test_one_pass_kernel_block_shapes(oracle, C, T, R):
+    d, x, y, sens, mask = problem(2, 1, C, T, (1, R, 160), MASK_READOUT_INVARIANT, sens_has_frames=1, seed=C + T, density=0.14)
+    check(oracle, d, x, y, sens, mask, 0.7, what="one-pass kernel, %d coils, %d frames of %d rows" % (C, T, R))

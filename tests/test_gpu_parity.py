@@ -127,6 +127,7 @@ def test_unsampled_measurements_are_never_read(oracle, rank, n, mask_kind):
 
 @pytest.mark.parametrize("case", [
     (2, 2, 8, 1, (1, 64, 160), MASK_READOUT_INVARIANT),      # one-pass 2-D kernel
+    (2, 1, 6, 20, (1, 192, 160), MASK_READOUT_INVARIANT),    # the same, one block per SM with a group split by coils
     (3, 1, 4, 1, (8, 64, 32), MASK_READOUT_INVARIANT),       # separable 3-D path
     (3, 1, 3, 1, (6, 20, 24), MASK_FULL),                    # general path
 ])

@@ -23,9 +23,11 @@ namespace gleam {
 template <class P, bool HAS_Z, bool SMW = false>
 struct WarpFlat {
     static constexpr int N = P::N, R0 = P::R0, RL = P::RL;
-    static constexpr bool ELIGIBLE = (P::S == 2) && (RL == 8 || RL == 16 || RL == 32) && (R0 < RL) && (N % 2 == 0);
+    // R0 < RL is where the plain kernel wastes lanes in the RL-point stages; R0 > RL (368 = 23 x 16) also fits: the
+    // R0-point butterflies then run on all lanes of the image-side stages and the RL-point ones on numbered units
+    static constexpr bool ELIGIBLE = (P::S == 2) && (RL == 8 || RL == 16 || RL == 32) && (R0 != RL) && (N % 2 == 0);
     static constexpr int LW = 32 / RL;                     // lines per warp
-    static constexpr int UPC = LW * R0;                    // k-space units per coil (< 32)
+    static constexpr int UPC = LW * R0;                    // k-space units per coil
     static constexpr int USTRIDE = RL + 1;                 // odd: a round's 32 units read without bank conflicts
     static constexpr int SLOTS_MIN = (32 + UPC - 1) / UPC + 1;     // coils between first forward and inverse stage
     // a ring whose unit count is a multiple of 16 keeps the bank pattern across the wrap; taken when small
@@ -63,7 +65,7 @@ struct WarpFlat {
 // with z).  A template parameter, not a run-time test of a.aty: with the test in the code the plain call measured
 // 11 % slower (17.7 against 16.0 us), although it never takes that branch.
 template <class P, bool HAS_Z, bool SMW, bool HAS_ATY>
-__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : (P::RL == 32 ? 12 : 16))
+__global__ void __launch_bounds__(SMW ? 512 : 32, SMW ? 1 : (P::R0 > 16 ? 8 : P::RL == 32 ? 12 : 16))
 warpflat_kernel(const RowArgs a, const int nwhole) {
     grid_dependency_wait();
     grid_launch_dependents();

@@ -116,7 +116,7 @@ inline cudaError_t launch_warpflat_zy(const RowArgs& a, cudaStream_t s) {
     // SM: the groups beyond 4 k are split by coils over four warps each, one per scheduler.  (Measured on cine-shaped
     // problems, per call: 13 groups per SM 18.7 -> 16.6 us, 12 per SM 18.7 -> 15.3 us; up to 7 per SM single-warp
     // blocks are faster, 11.3 against 12.7 us.)
-    if constexpr (P::RL <= 16) {        // 32-point butterflies need more registers than 16 warps per SM leave
+    if constexpr (P::RL <= 16 && P::R0 <= 12) {   // larger butterflies need more registers than 16 warps per SM leave
         using WS = WarpFlat<P, HAS_Z, true>;
         static PerDevice attrs_done;
         int sms = 0, dev = 0;
@@ -166,9 +166,11 @@ template <> struct FlatRL<192> { static constexpr int value = 32; };    // 6 x 3
 template <> struct FlatRL<96> { static constexpr int value = 16; };     // 6 x 16
 template <> struct FlatRL<80> { static constexpr int value = 16; };     // 5 x 16
 template <> struct FlatRL<48> { static constexpr int value = 8; };      // 6 x 8
-// lengths whose plain plan already keeps most lanes busy: the coil-numbered kernel only where it measured faster,
-// the call with z (192: forward 25 against 50 us, VJP 50 against 46 us on 8 x 16 coils x 512 rows)
-template <int N> struct FlatOnlyWithZ { static constexpr bool value = (N == 192); };
+template <> struct FlatRL<368> { static constexpr int value = 16; };    // 23 x 16
+// Which calls of a length take the coil-numbered kernel (1: without z, 2: with z): only where it measured faster.
+// 192: the plain plan already keeps most lanes busy (forward 25 against 50 us, but VJP 50 against 46 us on 8 x 16 coils x
+// 512 rows); 368 = 23 x 16 (252 registers, 8 warps per SM): VJP 84 against 96 us on knee2d, forward 158 against 153 us.
+template <int N> struct FlatCalls { static constexpr int value = (N == 192) ? 2 : (N == 368) ? 1 : 3; };
 template <class P> struct FlatPlan {
     static constexpr int RL = FlatRL<P::N>::value;
     using type = Plan<P::N, RL ? P::N / RL : P::R0, RL ? RL : P::R1, RL ? 1 : P::R2>;
@@ -180,7 +182,7 @@ inline cudaError_t launch_warpline(const RowArgs& a, cudaStream_t s) {
         using PF = typename FlatPlan<P>::type;
         static_assert(WarpFlat<PF, false>::ELIGIBLE, "not a plan the coil-numbered kernel takes");
         // the numbering across coils pays once a round of 32 units spans more than one coil
-        if (flat_enabled() && a.C >= 2 && (a.z != nullptr || !FlatOnlyWithZ<P::N>::value))
+        if (flat_enabled() && a.C >= 2 && (FlatCalls<P::N>::value & (a.z != nullptr ? 2 : 1)) != 0)
             return a.z != nullptr ? launch_warpflat_z<PF, true>(a, s) : launch_warpflat_z<PF, false>(a, s);
     }
     if (MODE == ROW_FUSED && a.z != nullptr) return launch_warpline_z<P, MODE, true>(a, s);

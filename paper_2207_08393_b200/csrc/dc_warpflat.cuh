@@ -61,7 +61,10 @@ struct WarpFlat {
 // coil sums are added in warp order through shared memory.  A quarter of the extra work lands on every scheduler.
 // One block per SM also keeps a dependent launch from moving in next to the running one warp by warp, which
 // would fill the schedulers unevenly.
-// HAS_ATY: the coil sum starts from minus the given A^H y image (normal-equations form of the step; never together
+// HAS_ATY: the coil sum is kept as aty - sum, starting from the given A^H y image as loaded (no instruction depends on
+// the load before the first inverse stage, so its latency is hidden even when a warp has a single group; the coil
+// terms are subtracted and the update adds eta times the result: the same bits as sum - aty, since rounding is
+// symmetric in the sign).  Normal-equations form of the step; never together
 // with z).  A template parameter, not a run-time test of a.aty: with the test in the code the plain call measured
 // 11 % slower (17.7 against 16.0 us), although it never takes that branch.
 template <class P, bool HAS_Z, bool SMW, bool HAS_ATY>
@@ -189,7 +192,7 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
 
         cf acc[R0];
 #pragma unroll
-        for (int m = 0; m < R0; ++m) acc[m] = (HAS_ATY && row_ok && q == 0) ? coil_sum_start(a.aty, x_off + j + RL * m) : make_float2(0.f, 0.f);
+        for (int m = 0; m < R0; ++m) acc[m] = (HAS_ATY && row_ok && q == 0) ? a.aty[x_off + j + RL * m] : make_float2(0.f, 0.f);
         cf sf[R0];                       // sensitivities of the next forward image-side stage
         if (nc > 0) load_sens(sf, 0);
         int af = 0, ai = 0;              // next coil of the forward / of the inverse image-side stage
@@ -287,8 +290,13 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
                 Dft<R0, +1>::run(v);
 #pragma unroll
                 for (int m = 0; m < R0; ++m) {
-                    acc[m].x = fmaf(si[m].x, v[m].x, fmaf(si[m].y, v[m].y, acc[m].x));
-                    acc[m].y = fmaf(si[m].x, v[m].y, fmaf(-si[m].y, v[m].x, acc[m].y));
+                    if (HAS_ATY) {      // acc = aty - sum
+                        acc[m].x = fmaf(-si[m].x, v[m].x, fmaf(-si[m].y, v[m].y, acc[m].x));
+                        acc[m].y = fmaf(-si[m].x, v[m].y, fmaf(si[m].y, v[m].x, acc[m].y));
+                    } else {
+                        acc[m].x = fmaf(si[m].x, v[m].x, fmaf(si[m].y, v[m].y, acc[m].x));
+                        acc[m].y = fmaf(si[m].x, v[m].y, fmaf(-si[m].y, v[m].x, acc[m].y));
+                    }
                 }
                 ++ai;
             }
@@ -317,7 +325,8 @@ warpflat_kernel(const RowArgs a, const int nwhole) {
             for (int m = 0; m < R0; ++m) {
                 const cf xv = x_at(j + RL * m);
                 const cf av = acc[m];
-                const cf ov = make_float2(fmaf(-a.eta, av.x, xv.x), fmaf(-a.eta, av.y, xv.y));
+                const float se = HAS_ATY ? a.eta : -a.eta;          // HAS_ATY: acc holds aty - sum
+                const cf ov = make_float2(fmaf(se, av.x, xv.x), fmaf(se, av.y, xv.y));
                 store_image(a.out, x_off + j + RL * m, ov, a.out_planar, b, a.plane);
                 if (a.dot_rows != nullptr) dsum += (double)xv.x * ov.x + (double)xv.y * ov.y;
             }

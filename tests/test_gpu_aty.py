@@ -28,6 +28,7 @@ def run_aty(d, x, aty, sens, mask, eta, in_place=False, alias_aty=False):
 
 CASES = [
     (2, 2, 5, 3, (1, 24, 160), MASK_READOUT_INVARIANT, 0),      # units numbered across coils, single-warp blocks
+    (2, 1, 5, 20, (1, 192, 160), MASK_READOUT_INVARIANT, 1),    # one block per SM, one group split over four warps (1, 1, 1, 2 coils)
     (2, 1, 4, 2, (1, 10, 64), MASK_READOUT_INVARIANT, 1),       # four lines per warp
     (2, 2, 3, 1, (1, 12, 320), MASK_READOUT_INVARIANT, 0),      # one line per warp
     (2, 1, 3, 1, (1, 6, 384), MASK_READOUT_INVARIANT, 0),       # three-stage plan: block-synchronised row kernel

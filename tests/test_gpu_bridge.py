@@ -13,7 +13,9 @@ pytestmark = pytest.mark.gpu
 CASES = [
     (2, 2, 3, 2, (1, 20, 48), MASK_READOUT_INVARIANT),      # one-pass 2-D kernel
     (2, 1, 2, 1, (1, 12, 46), MASK_READOUT_INVARIANT),      # line length 2 mod 4
-    (2, 1, 4, 1, (1, 16, 320), MASK_READOUT_INVARIANT),     # block-synchronised row kernel
+    (2, 1, 4, 1, (1, 16, 320), MASK_READOUT_INVARIANT),     # one line per warp, k-space units numbered across coils
+    (2, 1, 5, 20, (1, 192, 160), MASK_READOUT_INVARIANT),   # one block per SM with a group split by coils
+    (2, 1, 3, 1, (1, 8, 384), MASK_READOUT_INVARIANT),      # block-synchronised row kernel (three-stage plan)
     (2, 2, 3, 1, (1, 12, 16), MASK_FULL),
     (3, 2, 3, 1, (6, 64, 32), MASK_READOUT_INVARIANT),      # row-tile 3-D path
     (3, 1, 2, 2, (4, 46, 32), MASK_READOUT_INVARIANT),      # general 3-D path

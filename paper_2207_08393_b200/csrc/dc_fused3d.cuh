@@ -143,7 +143,12 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
     using namespace fused;
     constexpr int N1 = RY * BY;
     static_assert(BY >= 2 && BY <= 24 && BY % 2 == 0, "radix of the middle pass (even: the half shift of ky keeps ky mod RY)");
-    static_assert(BY * NZ * 8 + BY * NZ * 4 <= 2 * TILE * 8, "tile and mask rows of the middle pass fit buffers A | B");
+    // The mask rows of the middle pass arrive on buffer B's barrier and are guarded by B's release, so they have to
+    // lie in B's part of the shared memory: behind the tile rows that spill into B (BY > RY), else at B's start.  (At
+    // gbase + BY * NZ they lay inside buffer A for BY < RY, where a block that went from a third-pass item straight to a
+    // middle-pass item had them written over the partial coil sums still kept in A.)
+    constexpr int MASK_OFF = BY * NZ > TILE ? BY * NZ : TILE;
+    static_assert(MASK_OFF >= TILE && MASK_OFF * 8 + BY * NZ * 4 <= 2 * TILE * 8, "mask rows of the middle pass fit buffer B");
     extern __shared__ __align__(128) float2 fsmem[];
     float2* const smem = fsmem;
     Shared* sh = reinterpret_cast<Shared*>(smem + 2 * GROUP_ELEMS);
@@ -266,7 +271,7 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
                     if (bytes_b > 0) {
                         if (!(ok = begin_fill(1, bytes_b))) break;
                         if (ROWS_B > 0) bulk_load(gbase + TILE, src + ROWS_A * NZ, ROWS_B * NZ * 8, &sh->full[g][1]);
-                        if (s == 0) tma_load_4d(gbase + BY * NZ, &tm_mask, 0, k0, 0, bt, &sh->full[g][1]);
+                        if (s == 0) tma_load_4d(gbase + MASK_OFF, &tm_mask, 0, k0, 0, bt, &sh->full[g][1]);
                     }
                     if (!(ok = begin_fill(0, ROWS_A * NZ * 8))) break;
                     bulk_load(gbase, src, ROWS_A * NZ * 8, &sh->full[g][0]);
@@ -453,7 +458,7 @@ fused3d_kernel(const FusedArgs a, const __grid_constant__ CUtensorMap tm_sens, c
 #pragma unroll
                 for (int j = 0; j < BY; ++j) twy[j] = unit_root_fwd<N1>((j * k0) % N1);
                 float wts[BY];
-                const float* mrows = reinterpret_cast<const float*>(gbase + BY * NZ);
+                const float* mrows = reinterpret_cast<const float*>(gbase + MASK_OFF);
                 for (int s = 0; s < n; ++s) {
                     const int c = c_first + s;
                     wait_full(0);

@@ -157,15 +157,23 @@ struct Layout {
     int R, L2, L3;
 };
 
-// Ring size and lags of the fused kernel, in slabs: P2 follows P1 by L2 = 2 periods, P3 by L3 = 4, and the ring
-// holds R = 8 slabs (42 MB for 8 coils of 320 x 256).  Larger settings were timed faster on the 320 x 320 x 256
-// volume ((12, 3, 6) 2.04 ms, (16, 4, 8) 1.81 ms per VJP call against 2.36 ms), but with (16, 4, 8) a 16-slab problem
-// came back with whole slabs wrong in most runs (slabs 8 to 10, whose third pass is drawn while first-pass items are
-// already being skipped; cause not found by reading), so those timings are indicative only and no other setting
-// than the one all tests pass with can be selected.
-static void fused_ring(int* R, int* L2, int* L3) { *R = 8; *L2 = 2; *L3 = 4; }
-// The persistent kernel is opt-in: measured on the 320 x 320 x 256 volume it is slower than the three whole-volume
-// passes (2.36 ms against 1.77-1.85 ms per VJP call at the default ring), so the default keeps those.  GLEAM_FUSED=1 in the environment
+// Ring size and lags of the fused kernel, in slabs.  One block per SM is resident and a period of one slab has fewer
+// items than there are SMs, so three to four slabs are in flight per pass and a dependency is only surely met after
+// about four periods: P2 follows P1 by L2 = 4 periods, P3 by L3 = 8, and the ring holds R = 16 slabs (84 MB for 8
+// coils of 320 x 256).  Measured per VJP call on the 320 x 320 x 256 volume: (8, 2, 4) 2.36 ms, (12, 3, 6) 2.04 ms,
+// (16, 4, 8) 1.81 ms.  GLEAM_FUSED_RING="R,L2,L3" overrides (tuning aid, read once).
+static void fused_ring(int* R, int* L2, int* L3) {
+    static int v[3] = {0, 0, 0};
+    if (v[0] == 0) {
+        int r = 16, l2 = 4, l3 = 8;
+        const char* e = getenv("GLEAM_FUSED_RING");
+        if (e) { int a = 0, b = 0, c = 0; if (sscanf(e, "%d,%d,%d", &a, &b, &c) == 3 && a > c && c >= b && b >= 1 && a <= 64) { r = a; l2 = b; l3 = c; } }
+        v[1] = l2; v[2] = l3; v[0] = r;
+    }
+    *R = v[0]; *L2 = v[1]; *L3 = v[2];
+}
+// The persistent kernel is opt-in: measured on the 320 x 320 x 256 volume it only draws level with the three
+// whole-volume passes (1.81 ms against 1.77-1.93 ms per VJP call), so the default keeps those.  GLEAM_FUSED=1 in the environment
 // or gleam_dc_set_fused(1) selects it; the choice changes the workspace layout, so it is made before
 // gleam_dc_workspace_size.
 static std::atomic<int> g_fused_on{-1};

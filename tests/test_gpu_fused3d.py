@@ -39,8 +39,8 @@ def test_fused_path_matches_oracle(oracle, B, C, T, n):
 
 
 def test_fused_path_knee3d_full_size_vjp(oracle):
-    """The whole 320 x 320 x 256 volume with 8 coils through the persistent kernel (320 slabs, 40 turns of the default
-    ring of 8 slabs), element by element against the oracle; the status word stays clear."""
+    """The whole 320 x 320 x 256 volume with 8 coils through the persistent kernel (320 slabs, 20 turns of the default
+    ring of 16 slabs), element by element against the oracle; the status word stays clear."""
     import torch
     import paper_2207_08393_b200 as g
     from oracle.oracle import Dims
@@ -81,6 +81,19 @@ def test_fused_path_is_deterministic():
     for _ in range(20):
         assert np.array_equal(first, run_gpu(x, None, sens, mask, 1.0, 3, 0, MASK_READOUT_INVARIANT))
         assert np.array_equal(first_f, run_gpu(x, y, sens, mask, 1.0, 3, 0, MASK_READOUT_INVARIANT))
+
+
+@pytest.mark.parametrize("n", [(16, 64, 256), (12, 128, 256)])
+def test_fused_path_repeats_with_a_small_middle_radix(oracle, n):
+    """Planes of 64 and 128 rows (middle radix 4 and 8, below the 16 rows of a tile): the mask rows of a middle-pass
+    item share a buffer with nothing else that is live.  A block that goes from a third-pass item straight to a
+    middle-pass item whose dependency is already met is the case that once wrote them over live partial sums, now
+    and then: ten runs each, every one against the oracle."""
+    d, x, y, sens, mask = problem(3, 1, 5, 1, n, MASK_READOUT_INVARIANT, seed=sum(n), density=0.15)
+    ref = oracle.dc_vjp(x, sens, mask, 1.0, d, nthreads=8)
+    for i in range(10):
+        got = run_gpu(x, None, sens, mask, 1.0, 3, 0, MASK_READOUT_INVARIANT)
+        assert_close(got, ref, x, "fused vjp %s, run %d" % (n, i))
 
 
 def test_status_is_ok_after_a_normal_call():
